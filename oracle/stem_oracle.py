@@ -1,0 +1,148 @@
+"""CPU checker for the STEM FFN layer (test infrastructure, not a product path).
+
+A plain fp64 numpy statement of what the layer computes, written from the paper's
+definition.  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+import this file; nothing in the CUDA path does, and it imports nothing from that path.
+It is deliberately unblocked and unfused so it can be read against the equations:
+
+* forward   -- Section 3.1 (STEM), the layer equation
+              y = W_d ( SiLU(W_g x) (.) U[t] ),
+              with the matrix orientations of Section 2 (Background):
+              W_g in R^{d_ff x d}, W_d in R^{d x d_ff}, U in R^{V x d_ff}.
+* backward  -- the paper gives no formulas (it only says training sends the table's
+              gradients back, Table 1 notes); these are the chain rule of the forward
+              for the loss  L = sum_{t,i} dy[t,i] * y[t,i].
+* dedup     -- the paper only names token deduplication (Section 3.3); the arrays are
+              defined here: positions stably sorted by id, the distinct ids ascending,
+              where each id's run starts, and each position's slot.
+
+SiLU is not defined in the paper; the standard SiLU(z) = z * sigmoid(z) is used.
+Token ids are 0-based.  There are no bias terms (Table 1 caption).
+
+Pins (tests/test_oracle_pins.py): dense SwiGLU on one-hot augmented input through
+torch autograd, central finite differences, brute-force per-id sums and index arrays,
+special values, permutation equivariance.  Every function here has at least one pin.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def sigmoid(z: np.ndarray) -> np.ndarray:
+    return 1.0 / (1.0 + np.exp(-z))
+
+
+def silu(z: np.ndarray) -> np.ndarray:
+    """SiLU(z) = z * sigmoid(z)."""
+    return z * sigmoid(z)
+
+
+def silu_grad(z: np.ndarray) -> np.ndarray:
+    """d/dz SiLU(z) = sigmoid(z) * (1 + z * (1 - sigmoid(z)))."""
+    s = sigmoid(z)
+    return s * (1.0 + z * (1.0 - s))
+
+
+def _f64(a) -> np.ndarray:
+    return np.asarray(a, dtype=np.float64)
+
+
+def forward(x, ids, W_gate, E, W_down, return_intermediates: bool = False):
+    """Section 3.1, the STEM layer equation, for every position t.
+
+    x [T,d], ids [T] int, W_gate [F,d], E [V,F], W_down [d,F]  ->  y [T,d].
+    """
+    x, W_gate, W_down = _f64(x), _f64(W_gate), _f64(W_down)
+    ids = np.asarray(ids, dtype=np.int64)
+    G = x @ W_gate.T                    # g_t = W_g x_t
+    A = silu(G)                         # SiLU(g_t)
+    U = _f64(E[ids])                    # U[t], the looked-up row
+    H = A * U                           # SiLU(g_t) (.) U[t]
+    y = H @ W_down.T                    # y_t = W_d h_t
+    if return_intermediates:
+        return y, {"G": G, "A": A, "U": U, "H": H}
+    return y
+
+
+def dedup(ids):
+    """Index arrays of token deduplication (Section 3.3 names the step only).
+
+    perm        : positions sorted by (ids[t], t) ascending  -- a stable sort by id
+    unique_ids  : the distinct ids, ascending
+    seg_offsets : seg_offsets[r] = first index in perm of unique_ids[r]; last entry = T
+    inverse     : inverse[t] = r  with  unique_ids[r] == ids[t]
+    """
+    ids = np.asarray(ids, dtype=np.int64)
+    T = ids.shape[0]
+    perm = np.lexsort((np.arange(T), ids))
+    sorted_ids = ids[perm]
+    is_head = np.ones(T, dtype=bool)
+    is_head[1:] = sorted_ids[1:] != sorted_ids[:-1]
+    heads = np.flatnonzero(is_head)
+    unique_ids = sorted_ids[heads]
+    seg_offsets = np.concatenate([heads, [T]])
+    slot_of_sorted = np.cumsum(is_head) - 1
+    inverse = np.empty(T, dtype=np.int64)
+    inverse[perm] = slot_of_sorted
+    return {
+        "perm": perm.astype(np.int32),
+        "unique_ids": unique_ids.astype(np.int32),
+        "seg_offsets": seg_offsets.astype(np.int32),
+        "inverse": inverse.astype(np.int32),
+        "n_unique": int(unique_ids.shape[0]),
+    }
+
+
+def backward(dy, x, ids, W_gate, E, W_down):
+    """Chain rule of `forward` for L = sum dy * y.
+
+    Returns dx [T,d], dW_gate [F,d], dW_down [d,F], and the table gradient in compact
+    form: unique_ids [n_u] ascending and dE_rows [n_u,F] with
+    dE_rows[r] = sum over positions t with ids[t] == unique_ids[r] of dU[t]
+    (rows of E that no position uses have zero gradient and no row here).
+    """
+    dy, x, W_gate, W_down = _f64(dy), _f64(x), _f64(W_gate), _f64(W_down)
+    ids = np.asarray(ids, dtype=np.int64)
+    _, im = forward(x, ids, W_gate, E, W_down, return_intermediates=True)
+    G, A, U, H = im["G"], im["A"], im["U"], im["H"]
+
+    dH = dy @ W_down                    # dh_t = W_d^T dy_t
+    dW_down = dy.T @ H                  # sum_t dy_t h_t^T
+    dU = dH * A                         # dL/dU[t] contribution of position t
+    dA = dH * U
+    dG = dA * silu_grad(G)
+    dW_gate = dG.T @ x                  # sum_t dg_t x_t^T
+    dx = dG @ W_gate                    # W_g^T dg_t
+
+    unique_ids = np.unique(ids)
+    dE_rows = np.zeros((unique_ids.shape[0], dU.shape[1]), dtype=np.float64)
+    for r, v in enumerate(unique_ids):
+        dE_rows[r] = dU[ids == v].sum(axis=0)
+    return {
+        "dx": dx, "dW_gate": dW_gate, "dW_down": dW_down,
+        "unique_ids": unique_ids.astype(np.int32), "dE_rows": dE_rows,
+        "dU": dU, "dG": dG, "dH": dH,
+    }
+
+
+def dE_dense(unique_ids, dE_rows, V: int) -> np.ndarray:
+    """Scatter the compact table gradient into a [V,F] array (absent ids stay zero)."""
+    out = np.zeros((V, dE_rows.shape[1]), dtype=np.float64)
+    out[np.asarray(unique_ids, dtype=np.int64)] = dE_rows
+    return out
+
+
+def prefetch_rows(unique_ids, n_ids: int, host_E) -> np.ndarray:
+    """Row cache of the offloaded-table path (Section 3.3; Figure 1(c)):
+    cache[r] = E[unique_ids[r]] for r < n_ids."""
+    idx = np.asarray(unique_ids[:n_ids], dtype=np.int64)
+    return np.asarray(host_E)[idx].copy()
+
+
+def scaled_max_err(got, ref) -> float:
+    """max |got - ref| / max |ref|  -- the error measure the parity tests use."""
+    got, ref = _f64(got), _f64(ref)
+    denom = float(np.max(np.abs(ref))) if ref.size else 1.0
+    if denom == 0.0:
+        denom = 1.0
+    return float(np.max(np.abs(got - ref))) / denom if ref.size else 0.0

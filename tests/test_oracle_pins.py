@@ -1,0 +1,269 @@
+"""Pins for the CPU checker: each check compares oracle/stem_oracle.py with something
+that is not itself -- torch autograd on a textbook dense SwiGLU, finite differences,
+brute-force loops over positions, closed-form special values."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import stem_oracle as O
+from paper_2601_10639_b200 import synth
+
+
+def _rand_case(T=7, d=5, F=6, V=4, seed=0, dist="uniform"):
+    rng = np.random.default_rng(seed)
+    return dict(
+        x=rng.normal(size=(T, d)), dy=rng.normal(size=(T, d)),
+        W_gate=rng.normal(size=(F, d)) / np.sqrt(d), W_down=rng.normal(size=(d, F)) / np.sqrt(F),
+        E=rng.normal(size=(V, F)), ids=rng.integers(0, V, size=T) if dist == "uniform" else np.zeros(T, int),
+    )
+
+
+def _dense_swiglu_autograd(c):
+    """Background, Eq. (1): dense SwiGLU on [x ; onehot(id)] with block weights
+    W_g' = [W_gate 0], W_u' = [0 E^T], W_d' = W_down, differentiated by torch autograd."""
+    T, d = c["x"].shape
+    V, F = c["E"].shape
+    x = torch.tensor(c["x"], dtype=torch.float64, requires_grad=True)
+    Wg = torch.tensor(c["W_gate"], dtype=torch.float64, requires_grad=True)
+    Wd = torch.tensor(c["W_down"], dtype=torch.float64, requires_grad=True)
+    Et = torch.tensor(c["E"].T.copy(), dtype=torch.float64, requires_grad=True)     # W_u' block [F,V]
+    onehot = torch.nn.functional.one_hot(torch.tensor(c["ids"], dtype=torch.int64), V).to(torch.float64)
+    xa = torch.cat([x, onehot], dim=1)                                     # [T, d+V]
+    Wg_aug = torch.cat([Wg, torch.zeros(F, V, dtype=torch.float64)], dim=1)
+    Wu_aug = torch.cat([torch.zeros(F, d, dtype=torch.float64), Et], dim=1)
+    y = torch.nn.functional.linear(
+        torch.nn.functional.silu(torch.nn.functional.linear(xa, Wg_aug)) * torch.nn.functional.linear(xa, Wu_aug), Wd)
+    (y * torch.tensor(c["dy"], dtype=torch.float64)).sum().backward()
+    return dict(y=y.detach().numpy(), dx=x.grad.numpy(), dW_gate=Wg.grad.numpy(), dW_down=Wd.grad.numpy(),
+                dE=Et.grad.numpy().T)
+
+
+@pytest.mark.parametrize("seed,T,d,F,V", [(0, 7, 5, 6, 4), (1, 33, 16, 24, 9), (2, 64, 8, 40, 100)])
+def test_p1_reduces_to_dense_swiglu_autograd(seed, T, d, F, V):
+    c = _rand_case(T, d, F, V, seed)
+    ref = _dense_swiglu_autograd(c)
+    y = O.forward(c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    b = O.backward(c["dy"], c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    np.testing.assert_allclose(y, ref["y"], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(b["dx"], ref["dx"], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(b["dW_gate"], ref["dW_gate"], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(b["dW_down"], ref["dW_down"], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(O.dE_dense(b["unique_ids"], b["dE_rows"], V), ref["dE"], rtol=1e-11, atol=1e-12)
+
+
+def test_p6_central_finite_differences():
+    c = _rand_case(5, 4, 6, 3, seed=3)
+    b = O.backward(c["dy"], c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    dE = O.dE_dense(b["unique_ids"], b["dE_rows"], 3)
+
+    def loss(**over):
+        a = dict(c, **over)
+        return float((a["dy"] * O.forward(a["x"], a["ids"], a["W_gate"], a["E"], a["W_down"])).sum())
+
+    eps = 1e-5
+    for name, grad in (("x", b["dx"]), ("W_gate", b["dW_gate"]), ("W_down", b["dW_down"]), ("E", dE)):
+        base = c[name]
+        num = np.zeros_like(base)
+        for idx in itertools.product(*map(range, base.shape)):
+            p, m = base.copy(), base.copy()
+            p[idx] += eps
+            m[idx] -= eps
+            num[idx] = (loss(**{name: p}) - loss(**{name: m})) / (2 * eps)
+        np.testing.assert_allclose(grad, num, rtol=2e-7, atol=2e-8, err_msg=name)
+
+
+def test_forward_matches_per_token_python_loops():
+    """The layer equation written out position by position with scalar loops."""
+    import math
+    c = _rand_case(6, 3, 5, 4, seed=4)
+    y = O.forward(c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    for t in range(6):
+        h = []
+        for j in range(5):
+            g = sum(c["W_gate"][j, k] * c["x"][t, k] for k in range(3))
+            h.append(g / (1.0 + math.exp(-g)) * c["E"][c["ids"][t], j])
+        for i in range(3):
+            assert abs(sum(c["W_down"][i, j] * h[j] for j in range(5)) - y[t, i]) < 1e-12
+
+
+def test_p2_identical_x_and_ids_is_a_dense_swiglu():
+    """Every position identical: the up-projection W_u = u x0^T / |x0|^2 gives W_u x0 = u,
+    so the layer equals Eq. (1) with that W_u."""
+    c = _rand_case(9, 6, 8, 5, seed=5)
+    x0 = c["x"][0]
+    c["x"] = np.tile(x0, (9, 1))
+    c["ids"] = np.full(9, 3)
+    u = c["E"][3]
+    W_u = np.outer(u, x0) / (x0 @ x0)
+    xt = torch.tensor(c["x"])
+    ref = torch.nn.functional.linear(
+        torch.nn.functional.silu(torch.nn.functional.linear(xt, torch.tensor(c["W_gate"])))
+        * torch.nn.functional.linear(xt, torch.tensor(W_u)), torch.tensor(c["W_down"])).numpy()
+    np.testing.assert_allclose(O.forward(c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"]), ref, rtol=1e-11, atol=1e-13)
+    # identical x but varying ids: row t is the dense SwiGLU whose up-projection output is E[ids[t]]
+    c["ids"] = np.array([0, 1, 2, 3, 4, 0, 1, 2, 3])
+    y = O.forward(c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    a = torch.nn.functional.silu(torch.tensor(c["W_gate"] @ x0)).numpy()
+    for t in range(9):
+        np.testing.assert_allclose(y[t], c["W_down"] @ (a * c["E"][c["ids"][t]]), rtol=1e-11, atol=1e-13)
+
+
+def test_p3_p4_table_gradient_rows():
+    c = _rand_case(40, 4, 6, 12, seed=6)
+    c["ids"][c["ids"] == 7] = 2                      # make id 7 absent
+    b = O.backward(c["dy"], c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    dense = O.dE_dense(b["unique_ids"], b["dE_rows"], 12)
+    assert 7 not in set(b["unique_ids"].tolist())
+    assert np.all(dense[7] == 0.0)
+    # brute force: O(T * n_u) scan, position by position, using per-position dU from autograd-free algebra
+    dU = (c["dy"] @ c["W_down"]) * (lambda g: g / (1 + np.exp(-g)))(c["x"] @ c["W_gate"].T)
+    for r, v in enumerate(b["unique_ids"]):
+        acc = np.zeros(6)
+        for t in range(40):
+            if c["ids"][t] == v:
+                acc += dU[t]
+        np.testing.assert_allclose(b["dE_rows"][r], acc, rtol=1e-12, atol=1e-13)
+    for v in range(12):
+        if v not in set(c["ids"].tolist()):
+            assert np.all(dense[v] == 0.0)
+
+
+def test_p5_permuting_positions():
+    c = _rand_case(25, 5, 7, 6, seed=7)
+    rng = np.random.default_rng(70)
+    p = rng.permutation(25)
+    y = O.forward(c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    b = O.backward(c["dy"], c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    y2 = O.forward(c["x"][p], c["ids"][p], c["W_gate"], c["E"], c["W_down"])
+    b2 = O.backward(c["dy"][p], c["x"][p], c["ids"][p], c["W_gate"], c["E"], c["W_down"])
+    np.testing.assert_allclose(y2, y[p], rtol=1e-13)
+    np.testing.assert_allclose(b2["dx"], b["dx"][p], rtol=1e-13)
+    for k in ("dW_gate", "dW_down", "dE_rows"):
+        np.testing.assert_allclose(b2[k], b[k], rtol=1e-10, atol=1e-12)
+    d1, d2 = O.dedup(c["ids"]), O.dedup(c["ids"][p])
+    assert np.array_equal(d1["unique_ids"], d2["unique_ids"])
+    assert np.array_equal(d1["seg_offsets"], d2["seg_offsets"])
+
+
+def test_p7_special_values():
+    c = _rand_case(10, 4, 6, 5, seed=8)
+    assert O.silu(np.array([0.0]))[0] == 0.0
+    assert O.silu_grad(np.array([0.0]))[0] == 0.5
+    # published closed-form values: SiLU(1) = 1/(1+e^-1), SiLU'(1) = s(1 + (1 - s)), s = sigmoid(1)
+    s1 = 0.7310585786300049
+    assert abs(O.silu(np.array([1.0]))[0] - s1) < 1e-15
+    assert abs(O.silu_grad(np.array([1.0]))[0] - s1 * (2 - s1)) < 1e-15
+    assert abs(O.silu(np.array([-30.0]))[0]) < 1e-11 and abs(O.silu(np.array([30.0]))[0] - 30.0) < 1e-11
+    # W_gate = 0: y = 0, dE = 0, dW_down = 0, dg = dh * u / 2
+    z = np.zeros_like(c["W_gate"])
+    assert np.all(O.forward(c["x"], c["ids"], z, c["E"], c["W_down"]) == 0)
+    b = O.backward(c["dy"], c["x"], c["ids"], z, c["E"], c["W_down"])
+    assert np.all(b["dE_rows"] == 0) and np.all(b["dW_down"] == 0)
+    np.testing.assert_allclose(b["dG"], 0.5 * (c["dy"] @ c["W_down"]) * c["E"][c["ids"]], rtol=1e-13)
+    # E = 1: plain gated MLP without up-projection
+    ones = np.ones_like(c["E"])
+    ref = torch.nn.functional.silu(torch.tensor(c["x"] @ c["W_gate"].T)).numpy() @ c["W_down"].T
+    np.testing.assert_allclose(O.forward(c["x"], c["ids"], c["W_gate"], ones, c["W_down"]), ref, rtol=1e-12)
+    # linear in E and in W_down
+    y = O.forward(c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    np.testing.assert_allclose(O.forward(c["x"], c["ids"], c["W_gate"], -3 * c["E"], c["W_down"]), -3 * y, rtol=1e-12)
+    np.testing.assert_allclose(O.forward(c["x"], c["ids"], c["W_gate"], c["E"], 2 * c["W_down"]), 2 * y, rtol=1e-12)
+
+
+def _brute_dedup(ids):
+    T = len(ids)
+    uniq = sorted(set(int(v) for v in ids))
+    perm = sorted(range(T), key=lambda t: (int(ids[t]), t))
+    # rank counting, O(T^2): position of t in the sorted order
+    rank = [sum(1 for s in range(T) if (ids[s], s) < (ids[t], t)) for t in range(T)]
+    assert [perm[rank[t]] for t in range(T)] == list(range(T))
+    seg = [sum(1 for t in range(T) if ids[t] < v) for v in uniq] + [T]
+    inv = [uniq.index(int(ids[t])) for t in range(T)]
+    return uniq, perm, seg, inv
+
+
+@pytest.mark.parametrize("dist,T,V", [("uniform", 50, 9), ("zipf", 200, 64), ("same", 17, 5), ("distinct", 30, 40),
+                                      ("mix", 120, 33), ("uniform", 1, 3)])
+def test_p8_p9_index_arrays_vs_brute_force(dist, T, V):
+    ids = synth.token_ids(11, T, V, dist)
+    d = O.dedup(ids)
+    uniq, perm, seg, inv = _brute_dedup(ids.tolist())
+    assert d["unique_ids"].tolist() == uniq
+    assert d["perm"].tolist() == perm
+    assert d["seg_offsets"].tolist() == seg
+    assert d["inverse"].tolist() == inv
+    assert d["n_unique"] == len(uniq)
+    assert sum(seg[r + 1] - seg[r] for r in range(len(uniq))) == T
+    if dist == "same":
+        assert d["n_unique"] == 1 and d["seg_offsets"].tolist() == [0, T]
+    if dist == "distinct":
+        assert d["n_unique"] == T and d["perm"].tolist() == np.argsort(ids, kind="stable").tolist()
+
+
+def test_p8_table_gradient_edge_cases():
+    c = _rand_case(12, 4, 6, 20, seed=9)
+    c["ids"] = np.full(12, 5)
+    b = O.backward(c["dy"], c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    assert b["unique_ids"].tolist() == [5]
+    np.testing.assert_allclose(b["dE_rows"][0], b["dU"].sum(axis=0), rtol=1e-13)
+    c["ids"] = np.array([19, 3, 7, 0, 11, 2, 13, 5, 17, 1, 4, 9])
+    b = O.backward(c["dy"], c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    np.testing.assert_allclose(b["dE_rows"], b["dU"][np.argsort(c["ids"])], rtol=1e-13)
+
+
+def test_prefetch_rows_is_a_row_copy():
+    rng = np.random.default_rng(1)
+    E = rng.normal(size=(10, 4))
+    u = np.array([1, 4, 9, 0, 0], dtype=np.int32)
+    cache = O.prefetch_rows(u, 3, E)
+    assert cache.shape == (3, 4)
+    for r in range(3):
+        assert np.array_equal(cache[r], E[u[r]])
+
+
+def test_planted_mistakes_are_caught(monkeypatch):
+    """A dropped term, a wrong sign and a transposed operand in the checker each break a pin."""
+    c = _rand_case(9, 5, 6, 4, seed=12)
+    ref = _dense_swiglu_autograd(c)
+
+    def run():
+        y = O.forward(c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+        b = O.backward(c["dy"], c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+        ok = np.allclose(y, ref["y"], rtol=1e-10, atol=1e-12)
+        for k in ("dx", "dW_gate", "dW_down"):
+            ok = ok and np.allclose(b[k], ref[k], rtol=1e-10, atol=1e-12)
+        return ok and np.allclose(O.dE_dense(b["unique_ids"], b["dE_rows"], 4), ref["dE"], rtol=1e-10, atol=1e-12)
+
+    assert run()
+    good_grad = O.silu_grad
+    monkeypatch.setattr(O, "silu_grad", lambda z: O.sigmoid(z))                      # dropped term
+    assert not run()
+    monkeypatch.setattr(O, "silu_grad", lambda z: O.sigmoid(z) * (1 - z * (1 - O.sigmoid(z))))   # wrong sign
+    assert not run()
+    monkeypatch.setattr(O, "silu_grad", good_grad)
+    monkeypatch.setattr(O, "sigmoid", lambda z: 1.0 / (1.0 + np.exp(z)))             # sign inside sigmoid
+    assert not run()
+
+
+def test_synth_is_seeded_and_shaped():
+    w = synth.WORKLOADS["tiny_fp32"]
+    a, b = synth.make_inputs(w), synth.make_inputs(w)
+    for k in a:
+        assert np.array_equal(a[k], b[k])
+    assert a["x"].shape == (256, 256) and a["E"].shape == (4096, 688) and a["ids"].dtype == np.int32
+    assert abs(a["x"].std() - 1.0) < 0.02 and abs(a["E"].std() - 0.02) < 0.001
+    assert abs(a["W_gate"].std() - 256 ** -0.5) < 0.002 and abs(a["W_down"].std() - 688 ** -0.5) < 0.002
+    # any slice regenerates alone
+    part = synth.normal(synth.BASE_SEED, synth.TAG_X, (256, 256))[3, 5:9]
+    assert np.array_equal(a["x"][3, 5:9], part)
+    # Zipf(1.1) over 32000 ids, 16384 draws: about 3.8k distinct ids, hottest id ~14 % of positions
+    ids = synth.token_ids(synth.BASE_SEED, 16384, 32000, "zipf")
+    n_u = len(np.unique(ids))
+    assert 3500 < n_u < 4200
+    assert 0.12 < np.mean(ids == 0) < 0.16
+    mix = synth.token_ids(synth.BASE_SEED, 32768, 32000, "mix")
+    assert 9500 < len(np.unique(mix)) < 11000
+    r = synth.round_bf16(a["x"])
+    assert np.array_equal(synth.round_bf16(r), r) and np.max(np.abs(r - a["x"]) / np.abs(a["x"])) <= 2.0 ** -8
