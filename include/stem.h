@@ -1,0 +1,176 @@
+/*
+ * libstem -- the STEM feed-forward layer on NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The layer (paper Section 3.1, "STEM", the layer equation):
+ *
+ *     y_t = W_down ( SiLU(W_gate x_t) (.) E[id_t] )          for every position t
+ *
+ * with W_gate in R^{d_ff x d_model}, W_down in R^{d_model x d_ff} (orientations of
+ * Section 2, "Background") and a layer-local table E in R^{V x d_ff} (the paper's U_l)
+ * that replaces the dense up-projection of a SwiGLU block.  SiLU(z) = z * sigmoid(z);
+ * no bias terms (Table 1 caption); token ids are 0-based.
+ *
+ * Conventions shared by every entry point
+ *   - All matrices are dense row-major: x,y,dy,dx [T,d_model]; W_gate,dW_gate
+ *     [d_ff,d_model]; W_down,dW_down [d_model,d_ff]; E [V,d_ff]; G,H [T,d_ff].
+ *   - Unless a parameter says "host", pointers are device pointers, 16-byte aligned.
+ *     The caller owns every buffer, the workspace included.  The library allocates no
+ *     device memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *     only enqueue work; they do not synchronise unless stated.
+ *   - Outputs are overwritten, never accumulated into.
+ *   - Return value: STEM_OK or a negative STEM_ERR_* code.  Conditions only the device
+ *     can see (an id outside [0,V), a pipeline wait that ran out) are recorded in the
+ *     workspace's status word and read back with stem_query_status().  A bad id is
+ *     clamped into range so no access leaves the table.  Nothing traps, prints from the
+ *     device or throws; there is no CPU fallback.
+ *   - dtype 0: fp32 storage and fp32 FMA arithmetic.  dtype 1: bf16 storage, bf16
+ *     tensor-core products accumulated in fp32, elementwise math in fp32, results
+ *     rounded to bf16 (round to nearest even) when stored.
+ *   - Shape limits: T <= 2^22; d_model and d_ff multiples of 8 (bf16) or 4 (fp32);
+ *     V <= 2^30.  T = 0 is accepted by every call and does nothing.
+ */
+#ifndef STEM_H_
+#define STEM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define STEM_OK 0
+#define STEM_ERR_INVALID_ARG (-1)
+#define STEM_ERR_UNSUPPORTED_SHAPE (-2)
+#define STEM_ERR_UNSUPPORTED_ARCH (-3)
+#define STEM_ERR_WORKSPACE_TOO_SMALL (-4)
+#define STEM_ERR_NOT_PINNED (-5)
+#define STEM_ERR_CUDA (-6)
+#define STEM_ERR_TIMEOUT (-7)  /* device: a bounded pipeline wait expired          */
+#define STEM_ERR_ID_RANGE (-8) /* device: a token id was outside [0,V) (clamped)  */
+
+#define STEM_DTYPE_FP32 0
+#define STEM_DTYPE_BF16 1
+
+#define STEM_FLAG_SIMT 1 /* run the bf16 contractions on the plain-FMA kernels (debug aid) */
+
+typedef struct {
+  int32_t T;          /* positions in this call (batch x sequence)                 */
+  int32_t d_model;    /* d                                                          */
+  int32_t d_ff;       /* F                                                          */
+  int32_t V;          /* rows of E addressable by ids                               */
+  int32_t dtype;      /* STEM_DTYPE_*: x, y, dy, dx, W_gate, W_down, E, G, H        */
+  int32_t grad_dtype; /* STEM_DTYPE_*: dW_gate, dW_down, dE_rows                    */
+  int32_t flags;      /* STEM_FLAG_* bits                                           */
+} stem_shape_t;
+
+/* Library version, major*10000 + minor*100 + patch. */
+int stem_version(void);
+
+/* Text for a STEM_ERR_* code (static storage). */
+const char* stem_status_string(int code);
+
+/* Bytes of workspace that any call with this shape needs (the maximum over calls).
+ * The first 256 bytes of a workspace hold the status word. */
+int stem_workspace_bytes(const stem_shape_t* shape, size_t* bytes /*host, out*/);
+
+/* Clear the status word.  Call once after allocating a workspace (and to re-arm it
+ * after an error was read). */
+int stem_init_workspace(void* ws, size_t ws_bytes, void* stream);
+
+/* Synchronises `stream`, then copies the status word to *status_out (host):
+ * STEM_OK, STEM_ERR_TIMEOUT or STEM_ERR_ID_RANGE.  The word is sticky: the first
+ * error stays until stem_init_workspace(). */
+int stem_query_status(const void* ws, void* stream, int32_t* status_out /*host*/);
+
+/*
+ * Token deduplication (Section 3.3 "System Implementation": the batch's token ids are
+ * deduplicated so only uniq(B*L) rows move; Table 1, "Communication").  The paper
+ * names the step; the arrays are defined here, each with exactly one correct value:
+ *   perm[T]          positions sorted by (ids[t], t) ascending (stable radix sort by id)
+ *   unique_ids[n_u]  the distinct ids, ascending
+ *   seg_offsets[n_u+1]  index in perm where each id's run starts; seg_offsets[n_u] = T
+ *   inverse[T]       inverse[t] = r with unique_ids[r] == ids[t]
+ *   n_unique         device scalar n_u
+ * unique_ids needs room for min(T,V) entries, seg_offsets for min(T,V)+1.  `inverse`
+ * may be NULL.  Entries past n_u are left untouched.
+ */
+int stem_dedup_ids(const stem_shape_t* shape, const int32_t* ids, int32_t* unique_ids,
+                   int32_t* n_unique, int32_t* inverse, int32_t* perm, int32_t* seg_offsets,
+                   void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Forward (Section 3.1, the layer equation).  Two kernels:
+ *   G = x W_gate^T, H = SiLU(G) (.) E[ids]   -- the row lookup is fused in the GEMM's
+ *                                               epilogue; E[ids] is never materialised
+ *   y = H W_down^T
+ * G_save, H_save: optional [T,d_ff] outputs (dtype) kept for backward; either may be
+ * NULL (H then lives in the workspace).  With a prefetched row cache, pass
+ * ids := inverse and E := dev_cache with shape->V = rows of the cache.
+ */
+int stem_ffn_forward(const stem_shape_t* shape, const void* x, const int32_t* ids,
+                     const void* W_gate, const void* E, const void* W_down, void* y,
+                     void* G_save, void* H_save, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Backward.  The paper states no formulas (training is implied: Table 1 notes, Section
+ * 3.3); these are the chain rule of the layer equation for L = sum dy (.) y:
+ *   dH = dy W_down;  dU = dH (.) SiLU(G);  dG = dH (.) E[ids] (.) SiLU'(G)
+ *   dW_down = dy^T H;  dW_gate = dG^T x;  dx = dG W_gate
+ *   dE_rows[r] = sum of dU[t] over the positions t with ids[t] == unique_ids[r]
+ *                (fixed summation order: the result is bitwise reproducible)
+ * G_save, H_save: what stem_ffn_forward saved (required).  perm, seg_offsets, n_unique,
+ * unique_ids: from stem_dedup_ids on the same ids.  dE_rows [min(T,V), d_ff]
+ * (grad_dtype): rows >= n_u are left untouched; ids absent from the call have no row
+ * (their gradient is zero).  dW_gate, dW_down in grad_dtype; dx in dtype.  Any of dx,
+ * dW_gate, dW_down, dE_rows may be NULL to skip that output.
+ */
+int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, const int32_t* ids,
+                      const void* W_gate, const void* E, const void* W_down, const void* G_save,
+                      const void* H_save, const int32_t* perm, const int32_t* seg_offsets,
+                      const int32_t* n_unique, void* dx, void* dW_gate, void* dW_down,
+                      void* dE_rows, const int32_t* unique_ids, void* ws, size_t ws_bytes,
+                      void* stream);
+
+/*
+ * Row prefetch for a table kept off the device (Section 3.3: tables offloaded to CPU
+ * memory, rows of the deduplicated ids prefetched asynchronously with layer compute;
+ * Figure 1(c)):   dev_cache[r,:] = table[ids[r],:]   for r < *n_ids.
+ * table: [V,d_ff] (dtype) in page-locked host memory (cudaHostAlloc / cudaHostRegister;
+ * checked, else STEM_ERR_NOT_PINNED) or in device memory (a compact on-device gather).
+ * ids: device, normally unique_ids; n_ids: device scalar, so no host round trip is
+ * needed between dedup and prefetch.  dev_cache: device [min(T,V), d_ff].  Run it on a
+ * side stream to overlap the previous layer's GEMMs.
+ */
+int stem_prefetch_rows(const stem_shape_t* shape, const int32_t* ids, const int32_t* n_ids,
+                       const void* table, void* dev_cache, void* ws, void* stream);
+
+/*
+ * Gradient write-back for an off-device table (Table 1 notes: the table's gradients are
+ * transferred back to CPU for the optimizer update):
+ *   host_rows[r,:] = dE_rows[r,:] for r < *n_rows;  host_ids[r] = unique_ids[r];
+ *   *host_n = *n_rows.
+ * host_rows [min(T,V), d_ff] (grad_dtype), host_ids [min(T,V)], host_n [1]: page-locked
+ * host memory (checked).  The device writes them directly; they are complete once
+ * `stream` has been synchronised.
+ */
+int stem_writeback_rows(const stem_shape_t* shape, const void* dE_rows, const int32_t* unique_ids,
+                        const int32_t* n_rows, void* host_rows, int32_t* host_ids,
+                        int32_t* host_n, void* stream);
+
+/*
+ * Plain contraction on the same tensor-core kernel the layer uses (the y = H W_down^T
+ * step is exactly this; exposed for testing and reuse):
+ *   C[m,n] = sum_k A(m,k) B(n,k),  C row-major [M,N] (bf16 if c_fp32 == 0, else fp32).
+ * a_mn == 0: A stored [M,K] row-major (K contiguous); a_mn == 1: A stored [K,M]
+ * row-major (M contiguous).  b_mn likewise for B ([N,K] or [K,N]).  M, N, K multiples
+ * of 8.  bf16 inputs, fp32 accumulation.  ws: a workspace (status word only).
+ */
+int stem_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t a_mn, const void* B,
+                   int32_t b_mn, void* C, int32_t c_fp32, int32_t flags, void* ws, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STEM_H_ */

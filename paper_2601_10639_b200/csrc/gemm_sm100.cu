@@ -1,0 +1,388 @@
+// bf16 contraction on the 5th-generation tensor cores (tcgen05), fp32 accumulators in
+// tensor memory, operands staged by TMA -- with the layer's elementwise work fused into
+// the epilogue.
+//
+//   C[m,n] = sum_k A(m,k) B(n,k)
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 0      one thread issues TMA loads into a STAGES-deep shared-memory ring
+//   warp 1      allocates TMEM; one thread issues tcgen05.mma (128 x BN x 16 per
+//               instruction, four per 64-wide k block) and commits to mbarriers
+//   warps 2..5  epilogue: tcgen05.ld the finished 128 x BN fp32 tile (one row per thread),
+//               apply the fused elementwise step, store
+// Two accumulator tiles live in TMEM (2 x BN columns), so the epilogue of tile i overlaps
+// the MMAs of tile i+1.  Operands may be K-major or MN-major (the backward pass contracts
+// over the token dimension, which is the slow index of every [T, .] tensor); both use the
+// 128-byte swizzle, selected in the instruction and shared-memory descriptors.
+//
+// Every wait is bounded.  On expiry the role records STEM_ERR_TIMEOUT in the status word,
+// raises a CTA-wide abort flag, and all roles unwind: copies in flight are waited for
+// (again bounded), TMEM is freed, the kernel returns.
+#include <cuda.h>
+
+#include "ptx_sm100.cuh"
+#include "stem_internal.h"
+
+namespace stem {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int UMMA_K = 16;
+constexpr int kEpiWarps = 4;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr long long kWaitLimitCycles = 2000000000ll;  // ~1 s at boost clock
+constexpr int kAtomBytes = 64 * BK * 2;                // one 64(MN) x BK swizzled block
+
+template <int BN, int STAGES>
+struct Smem {
+  static constexpr int kABytes = BM * BK * 2;
+  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBarOffset = STAGES * kStageBytes;
+  // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain, tmem address, abort
+  static constexpr int kNumBars = 2 * STAGES + 5;
+  static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16 + 1024;  // + alignment slack
+};
+
+__device__ __forceinline__ float fast_sigmoid(float g) {
+  return __fdividef(1.0f, 1.0f + __expf(-g));
+}
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4& q, float (&v)[8]) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ uint4 pack_bf16x8(const float (&v)[8]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    w[i] = *reinterpret_cast<const uint32_t*>(&h);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Fused elementwise step on 32 consecutive columns of one output row.
+template <int KIND>
+__device__ __forceinline__ void epilogue_row32(const EpiParams& ep, bool row_ok, size_t row_off,
+                                               const __nv_bfloat16* e_row, int n, int N,
+                                               const uint32_t (&acc)[32]) {
+  if (!row_ok) return;
+#pragma unroll
+  for (int g8 = 0; g8 < 4; ++g8) {
+    const int nn = n + g8 * 8;
+    if (nn >= N) break;  // N is a multiple of 8: a group is wholly in or wholly out
+    float a[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = __uint_as_float(acc[g8 * 8 + i]);
+    if (KIND == kEpiStore) {
+      if (ep.out_fp32) {
+        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(ep.out) + row_off + nn);
+        dst[0] = make_float4(a[0], a[1], a[2], a[3]);
+        dst[1] = make_float4(a[4], a[5], a[6], a[7]);
+      } else {
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.out) + row_off + nn) = pack_bf16x8(a);
+      }
+    } else if (KIND == kEpiGate) {
+      float u[8], h[8];
+      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(e_row + nn)), u);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) h[i] = a[i] * fast_sigmoid(a[i]) * u[i];
+      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.H) + row_off + nn) = pack_bf16x8(h);
+      if (ep.G)
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.G) + row_off + nn) = pack_bf16x8(a);
+    } else {
+      float u[8], g[8], du[8], dg[8];
+      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(e_row + nn)), u);
+      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(ep.Gin) + row_off + nn)), g);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float s = fast_sigmoid(g[i]);
+        du[i] = a[i] * (g[i] * s);
+        dg[i] = a[i] * u[i] * (s * (1.0f + g[i] * (1.0f - s)));
+      }
+      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.H) + row_off + nn) = pack_bf16x8(du);
+      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.G) + row_off + nn) = pack_bf16x8(dg);
+    }
+  }
+}
+
+struct TileCoord { int m_blk, n_blk; };
+__device__ __forceinline__ TileCoord tile_coord(int tile, int tiles_m, int tiles_n, int group_m) {
+  const int per_group = group_m * tiles_n;
+  const int g = tile / per_group;
+  const int first_m = g * group_m;
+  const int gsize = min(group_m, tiles_m - first_m);
+  const int in = tile - g * per_group;
+  return {first_m + in % gsize, in / gsize};
+}
+
+template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               int M, int N, int K, int group_m, EpiParams ep) {
+  using L = Smem<BN, STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - raw);
+  const uint32_t bars = base + L::kBarOffset;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+  const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kBarOffset + L::kNumBars * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kBarOffset + L::kNumBars * 8 + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
+  const int num_tiles = tiles_m * tiles_n;
+  const int k_blocks = (K + BK - 1) / BK;
+  constexpr uint32_t kTmemCols = 2 * BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(tfull_bar(a), 1); ptx::mbar_init(tempty_bar(a), kEpiWarps); }
+    ptx::mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  int issued = 0;  // producer: k blocks handed to TMA so far
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const TileCoord tc = tile_coord(tile, tiles_m, tiles_n, group_m);
+        const int m0 = tc.m_blk * BM, n0 = tc.n_blk * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitCycles)) {
+            report_error(ep.status, STEM_ERR_TIMEOUT, 1);
+            *abort_flag = 1; ok = false; break;
+          }
+          const uint32_t a_dst = base + s * L::kStageBytes;
+          const uint32_t b_dst = a_dst + L::kABytes;
+          ptx::mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
+          const int k0 = kb * BK;
+          if (A_MN) {
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) ptx::tma_load_2d(a_dst + j * kAtomBytes, &tmA, full_bar(s), m0 + 64 * j, k0);
+          } else {
+            ptx::tma_load_2d(a_dst, &tmA, full_bar(s), k0, m0);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j) ptx::tma_load_2d(b_dst + j * kAtomBytes, &tmB, full_bar(s), n0 + 64 * j, k0);
+          } else {
+            ptx::tma_load_2d(b_dst, &tmB, full_bar(s), k0, n0);
+          }
+          ++issued;
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, BN, A_MN, B_MN);
+      int s = 0; uint32_t ph = 0;
+      int acc = 0; uint32_t aph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        if (!ptx::mbar_wait_bounded(tempty_bar(acc), aph ^ 1u, abort_flag, kWaitLimitCycles)) {
+          report_error(ep.status, STEM_ERR_TIMEOUT, 3);
+          *abort_flag = 1; ok = false; break;
+        }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitCycles)) {
+            report_error(ep.status, STEM_ERR_TIMEOUT, 2);
+            *abort_flag = 1; ok = false; break;
+          }
+          ptx::tc_fence_after();
+          const uint32_t a_src = base + s * L::kStageBytes;
+          const uint32_t b_src = a_src + L::kABytes;
+#pragma unroll
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            // K-major: 16 k elements = 32 bytes inside the 128-byte swizzled row; 8-row
+            // groups 1024 bytes apart.  MN-major: 16 k rows of 128 bytes; 64-wide MN blocks
+            // kAtomBytes apart, 8-row k groups 1024 bytes apart.
+            const uint64_t ad = A_MN ? ptx::make_smem_desc(a_src + kk * (UMMA_K * 128), kAtomBytes, 1024)
+                                     : ptx::make_smem_desc(a_src + kk * (UMMA_K * 2), 16, 1024);
+            const uint64_t bd = B_MN ? ptx::make_smem_desc(b_src + kk * (UMMA_K * 128), kAtomBytes, 1024)
+                                     : ptx::make_smem_desc(b_src + kk * (UMMA_K * 2), 16, 1024);
+            ptx::mma_bf16_ss(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
+          }
+          ptx::mma_commit(empty_bar(s));
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::mma_commit(tfull_bar(acc));
+        if (++acc == 2) { acc = 0; aph ^= 1u; }
+      }
+      if (!ok) {
+        // let MMAs already issued finish before TMEM is freed
+        ptx::mma_commit(drain_bar);
+        int zero = 0;
+        ptx::mbar_wait_bounded(drain_bar, 0, &zero, kWaitLimitCycles);
+      }
+    }
+  } else {
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    int acc = 0; uint32_t aph = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      const TileCoord tc = tile_coord(tile, tiles_m, tiles_n, group_m);
+      const int m = tc.m_blk * BM + q * 32 + lane;
+      const int n0 = tc.n_blk * BN;
+      const bool row_ok = m < M;
+      const size_t row_off = static_cast<size_t>(m) * N;
+      const __nv_bfloat16* e_row = nullptr;
+      if (KIND != kEpiStore && row_ok) {
+        int id = ep.ids[m];
+        if (id < 0 || id >= ep.V) {
+          report_error(ep.status, STEM_ERR_ID_RANGE, m);
+          id = id < 0 ? 0 : ep.V - 1;
+        }
+        e_row = static_cast<const __nv_bfloat16*>(ep.E) + static_cast<size_t>(id) * N;
+      }
+      bool mine = ptx::mbar_wait_bounded(tfull_bar(acc), aph, abort_flag, kWaitLimitCycles);
+      mine = __all_sync(0xffffffffu, mine);
+      if (!mine) {
+        if (lane == 0) { report_error(ep.status, STEM_ERR_TIMEOUT, 4); *abort_flag = 1; }
+        ok = false; break;
+      }
+      ptx::tc_fence_after();
+      const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(t_row + c * 32, v);
+        ptx::tmem_ld_wait();
+        epilogue_row32<KIND>(ep, row_ok, row_off, e_row, n0 + c * 32, N, v);
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; aph ^= 1u; }
+    }
+  }
+
+  __syncthreads();
+  if (*abort_flag != 0 && threadIdx.x == 0) {
+    // wait (bounded) for TMA copies still in flight: the last issue into each stage
+    int zero = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      int last = -1;
+      for (int j = issued - 1; j >= 0 && j >= issued - STAGES; --j)
+        if (j % STAGES == s) { last = j; break; }
+      if (last >= 0) ptx::mbar_wait_bounded(full_bar(s), (last / STAGES) & 1, &zero, kWaitLimitCycles / 16);
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                              CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                              CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode_fn() {
+  static EncodeFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeFn>(p);
+  }();
+  return fn;
+}
+
+// Row-major bf16 matrix [rows, cols] (cols contiguous); box = 64 columns x box_rows rows.
+bool encode_map(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows) {
+  EncodeFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+  const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES>
+cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, int M, int N, int K,
+                        const EpiParams& ep, cudaStream_t stream) {
+  using L = Smem<BN, STAGES>;
+  auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+  const int grid = tiles < device_sm_count() ? tiles : device_sm_count();
+  kern<<<grid, kThreads, L::kTotal, stream>>>(tmA, tmB, M, N, K, 8, ep);
+  return cudaGetLastError();
+}
+
+template <bool A_MN, bool B_MN, int KIND>
+cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const EpiParams& ep,
+                      cudaStream_t stream) {
+  constexpr int BN = 256, STAGES = 4;
+  CUtensorMap tmA, tmB;
+  const bool okA = A_MN ? encode_map(&tmA, A, K, M, BK) : encode_map(&tmA, A, M, K, BM);
+  const bool okB = B_MN ? encode_map(&tmB, B, K, N, BK) : encode_map(&tmB, B, N, K, BN);
+  if (!okA || !okB) return cudaErrorNotSupported;
+  return launch_inst<A_MN, B_MN, KIND, BN, STAGES>(tmA, tmB, M, N, K, ep, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const void* B, bool b_mn,
+                           EpiKind kind, const EpiParams& ep, cudaStream_t stream) {
+  if (M <= 0 || N <= 0) return cudaSuccess;
+  if (K <= 0 || (M % 8) || (N % 8) || (K % 8)) return cudaErrorNotSupported;
+  // layer call sites: gate (K,K,gate)  down (K,K,store)  dH (K,MN,dh)  dx (K,MN,store)
+  //                   dW_down / dW_gate (MN,MN,store); the plain-GEMM entry adds (MN,K,store)
+  if (!a_mn && !b_mn) {
+    if (kind == kEpiGate) return launch_bn<false, false, kEpiGate>(A, B, M, N, K, ep, stream);
+    if (kind == kEpiStore) return launch_bn<false, false, kEpiStore>(A, B, M, N, K, ep, stream);
+  } else if (!a_mn && b_mn) {
+    if (kind == kEpiDH) return launch_bn<false, true, kEpiDH>(A, B, M, N, K, ep, stream);
+    if (kind == kEpiStore) return launch_bn<false, true, kEpiStore>(A, B, M, N, K, ep, stream);
+  } else if (a_mn && b_mn) {
+    if (kind == kEpiStore) return launch_bn<true, true, kEpiStore>(A, B, M, N, K, ep, stream);
+  } else {
+    if (kind == kEpiStore) return launch_bn<true, false, kEpiStore>(A, B, M, N, K, ep, stream);
+  }
+  return cudaErrorNotSupported;
+}
+
+}  // namespace stem

@@ -1,0 +1,91 @@
+// Internal declarations shared by the translation units of libstem.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <cstddef>
+#include <cstdint>
+
+#include "../../include/stem.h"
+
+namespace stem {
+
+constexpr size_t kStatusBytes = 256;  // head of every workspace
+// status word layout (int32): [0] first error code, [1] detail, [2] count of bad ids
+struct StatusWord {
+  int32_t code;
+  int32_t detail;
+  int32_t bad_ids;
+};
+
+__device__ __forceinline__ void report_error(int32_t* status, int32_t code, int32_t detail) {
+  if (status == nullptr) return;
+  if (atomicCAS(status, 0, code) == 0) status[1] = detail;
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- element helpers ----------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) {
+  return __float2bfloat16_rn(v);
+}
+
+__device__ __forceinline__ float sigmoid_f32(float g) { return 1.0f / (1.0f + expf(-g)); }
+
+// ---- epilogue descriptions (shared by the FMA and the tensor-core GEMM front ends) ---
+enum EpiKind : int { kEpiStore = 0, kEpiGate = 1, kEpiDH = 2 };
+
+struct EpiParams {
+  // kEpiStore: out[m*ld + n] = acc              (out_fp32 selects fp32 or bf16/T storage)
+  void* out = nullptr;
+  int out_fp32 = 0;
+  // kEpiGate:  g = acc; H = SiLU(g) * E[ids[m], n]; optional G = g
+  // kEpiDH:    dh = acc; g = G[m,n]; u = E[ids[m], n];
+  //            dU = dh * SiLU(g); dG = dh * u * SiLU'(g)
+  const int32_t* ids = nullptr;
+  const void* E = nullptr;
+  int V = 0;
+  void* H = nullptr;    // kEpiGate: H out          kEpiDH: dU out
+  void* G = nullptr;    // kEpiGate: G out (opt.)   kEpiDH: dG out
+  const void* Gin = nullptr;  // kEpiDH: saved G
+  int32_t* status = nullptr;
+};
+
+// C[m,n] = sum_k A(m,k) B(n,k); a_mn/b_mn: operand stored with the M (N) index contiguous.
+// FMA-pipe kernels, any T in {float, bf16}; fp32 accumulation.
+cudaError_t launch_simt_gemm(int dtype, int M, int N, int K, const void* A, bool a_mn,
+                             const void* B, bool b_mn, EpiKind kind, const EpiParams& ep,
+                             cudaStream_t stream);
+
+// tcgen05 / TMEM / TMA kernels, bf16 inputs.  Returns cudaErrorNotSupported when the
+// shape cannot be described to TMA (the caller decides what to do).
+cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const void* B,
+                           bool b_mn, EpiKind kind, const EpiParams& ep, cudaStream_t stream);
+
+// ---- index path ----------------------------------------------------------------------
+size_t dedup_workspace_bytes(int T, int V);
+cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, int32_t* n_unique,
+                         int32_t* inverse, int32_t* perm, int32_t* seg_offsets, void* scratch,
+                         int32_t* status, cudaStream_t stream);
+
+// ---- table-gradient reduce --------------------------------------------------------------
+size_t segreduce_workspace_bytes(int T, int F);
+cudaError_t launch_segreduce(int T, int F, int in_dtype, int out_dtype, const void* dU,
+                             const int32_t* perm, const int32_t* seg_offsets,
+                             const int32_t* n_unique, void* dE_rows, void* scratch,
+                             cudaStream_t stream);
+
+// ---- row movers ---------------------------------------------------------------------------
+cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int32_t* ids,
+                               const int32_t* n_ids, const void* table, void* dst,
+                               int32_t* status, cudaStream_t stream);
+cudaError_t launch_writeback_rows(int max_rows, size_t row_bytes, const void* rows,
+                                  const int32_t* unique_ids, const int32_t* n_rows, void* host_rows,
+                                  int32_t* host_ids, int32_t* host_n, cudaStream_t stream);
+
+int device_sm_count();
+
+}  // namespace stem

@@ -1,0 +1,292 @@
+"""CUDA path vs the CPU checker, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import stem_oracle as O
+from paper_2601_10639_b200 import binding as B
+from paper_2601_10639_b200 import runner, synth
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32 = 1e-5   # scaled max-abs error, fp32 configuration
+TOL_BF16 = 2e-2   # bf16 inputs, fp32 accumulation
+
+
+def _np(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def _ws():
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    B.stem_init_workspace(ws)
+    return ws
+
+
+# ---------------------------------------------------------------------------------------
+# plain contraction, every operand layout, ragged tiles
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("flags", [0, B.FLAG_SIMT], ids=["tcgen05", "fma"])
+@pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 1), (1, 0)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (200, 328, 136), (512, 768, 1024), (8, 8, 8), (1000, 264, 520)])
+def test_gemm_layouts(flags, a_mn, b_mn, M, N, K):
+    rng = np.random.default_rng(M * 7 + N * 3 + K + a_mn * 2 + b_mn)
+    A = synth.round_bf16(rng.normal(size=(M, K)).astype(np.float32))
+    Bm = synth.round_bf16(rng.normal(size=(N, K)).astype(np.float32))
+    ref = A.astype(np.float64) @ Bm.astype(np.float64).T
+    dA = torch.from_numpy(np.ascontiguousarray(A.T if a_mn else A)).cuda().bfloat16()
+    dB = torch.from_numpy(np.ascontiguousarray(Bm.T if b_mn else Bm)).cuda().bfloat16()
+    ws = _ws()
+    for c_fp32 in (1, 0):
+        C = torch.full((M, N), float("nan"), dtype=torch.float32 if c_fp32 else torch.bfloat16, device="cuda")
+        B.stem_gemm_bf16(M, N, K, dA, a_mn, dB, b_mn, C, c_fp32, flags, ws)
+        assert B.stem_query_status(ws) == B.OK
+        err = O.scaled_max_err(_np(C), ref)
+        assert err <= (5e-5 if c_fp32 else 6e-3), (err, c_fp32)
+
+
+# ---------------------------------------------------------------------------------------
+# index path: bit exact
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dist,T,V", [
+    ("uniform", 256, 4096), ("zipf", 16384, 32000), ("mix", 32768, 32000), ("same", 1000, 77),
+    ("distinct", 3000, 5000), ("uniform", 1, 5), ("uniform", 70001, 300), ("zipf", 100000, 1 << 20),
+    ("uniform", 65, 2), ("uniform", 4097, 1),
+])
+def test_dedup_bit_exact(dist, T, V):
+    ids = synth.token_ids(5, T, V, dist)
+    ref = O.dedup(ids)
+    st = runner.LayerState(B.make_shape(T, 8, 8, V, B.DTYPE_BF16, B.DTYPE_FP32, 0)).allocate(backward=False)
+    st.ids = torch.from_numpy(ids).cuda()
+    st.bufs["unique_ids"].fill_(-7)
+    st.dedup()
+    assert st.status() == B.OK
+    n_u = int(st.bufs["n_unique"].item())
+    assert n_u == ref["n_unique"]
+    assert np.array_equal(st.bufs["unique_ids"][:n_u].cpu().numpy(), ref["unique_ids"])
+    assert np.array_equal(st.bufs["perm"][:T].cpu().numpy(), ref["perm"])
+    assert np.array_equal(st.bufs["seg_offsets"][:n_u + 1].cpu().numpy(), ref["seg_offsets"])
+    assert np.array_equal(st.bufs["inverse"][:T].cpu().numpy(), ref["inverse"])
+    if n_u < st.bufs["unique_ids"].numel():
+        assert int(st.bufs["unique_ids"][n_u].item()) == -7      # entries past n_u untouched
+
+
+def test_dedup_empty_and_bad_ids():
+    st = runner.LayerState(B.make_shape(0, 8, 8, 10, B.DTYPE_BF16, B.DTYPE_FP32, 0)).allocate(backward=False)
+    st.ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st.dedup()
+    assert int(st.bufs["n_unique"].item()) == 0 and int(st.bufs["seg_offsets"][0].item()) == 0
+    ids = np.array([3, 99, -4, 3, 0], dtype=np.int32)         # 99 and -4 are outside [0,10)
+    st = runner.LayerState(B.make_shape(5, 8, 8, 10, B.DTYPE_BF16, B.DTYPE_FP32, 0)).allocate(backward=False)
+    st.ids = torch.from_numpy(ids).cuda()
+    st.dedup()
+    assert st.status() == B.ERR_ID_RANGE
+    ref = O.dedup(np.clip(ids, 0, 9))
+    assert np.array_equal(st.bufs["perm"][:5].cpu().numpy(), ref["perm"])
+    B.stem_init_workspace(st.bufs["ws"])
+    assert st.status() == B.OK
+
+
+# ---------------------------------------------------------------------------------------
+# the layer, full comparison at sizes the checker finishes in seconds
+# ---------------------------------------------------------------------------------------
+def _full_parity(w, inputs, dtype_code, tol, flags=0, grad_dtype=B.DTYPE_FP32):
+    st = runner.state_from_numpy(inputs, dtype_code, w.V, grad_dtype=grad_dtype, flags=flags)
+    st.step()
+    torch.cuda.synchronize()
+    assert st.status() == B.OK
+    y_ref, im = O.forward(inputs["x"], inputs["ids"], inputs["W_gate"], inputs["E"], inputs["W_down"], True)
+    bw = O.backward(inputs["dy"], inputs["x"], inputs["ids"], inputs["W_gate"], inputs["E"], inputs["W_down"])
+    dd = O.dedup(inputs["ids"])
+    b = st.bufs
+    n_u = int(b["n_unique"].item())
+    assert n_u == dd["n_unique"]
+    assert np.array_equal(b["unique_ids"][:n_u].cpu().numpy(), dd["unique_ids"])
+    assert np.array_equal(b["perm"].cpu().numpy()[:w_T(inputs)], dd["perm"])
+    assert np.array_equal(b["seg_offsets"][:n_u + 1].cpu().numpy(), dd["seg_offsets"])
+    errs = {
+        "G": O.scaled_max_err(_np(b["G"]), im["G"]),
+        "H": O.scaled_max_err(_np(b["H"]), im["H"]),
+        "y": O.scaled_max_err(_np(b["y"]), y_ref),
+        "dx": O.scaled_max_err(_np(b["dx"]), bw["dx"]),
+        "dW_gate": O.scaled_max_err(_np(b["dW_gate"]), bw["dW_gate"]),
+        "dW_down": O.scaled_max_err(_np(b["dW_down"]), bw["dW_down"]),
+        "dE_rows": O.scaled_max_err(_np(b["dE_rows"][:n_u]), bw["dE_rows"]),
+    }
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, (bad, errs)
+    return st, errs
+
+
+def w_T(inputs):
+    return inputs["x"].shape[0]
+
+
+def test_layer_fp32_config():
+    """batch 2 x seq 128, d_model 256, d_ff 688, V 4096, fp32 throughout."""
+    w = synth.WORKLOADS["tiny_fp32"]
+    _full_parity(w, synth.make_inputs(w), B.DTYPE_FP32, TOL_FP32)
+
+
+@pytest.mark.parametrize("flags", [0, B.FLAG_SIMT], ids=["tcgen05", "fma"])
+@pytest.mark.parametrize("T,d,F,V,dist", [(300, 264, 520, 1000, "zipf"), (1024, 512, 768, 4096, "uniform"),
+                                          (130, 64, 72, 50, "same"), (257, 1024, 2816, 32000, "zipf")])
+def test_layer_bf16_small(flags, T, d, F, V, dist):
+    w = synth.Workload("t", T, d, F, V, "bf16", dist)
+    _full_parity(w, synth.make_inputs(w, seed=77), B.DTYPE_BF16, TOL_BF16, flags)
+
+
+def test_layer_bf16_grad_bf16():
+    w = synth.Workload("t", 512, 256, 512, 300, "bf16", "zipf")
+    _full_parity(w, synth.make_inputs(w, seed=78), B.DTYPE_BF16, TOL_BF16, 0, grad_dtype=B.DTYPE_BF16)
+
+
+def test_backward_is_bitwise_reproducible():
+    w = synth.Workload("t", 2048, 256, 1024, 500, "bf16", "zipf")
+    st = runner.state_from_numpy(synth.make_inputs(w, seed=79), B.DTYPE_BF16, w.V)
+    st.step()
+    torch.cuda.synchronize()
+    first = {k: st.bufs[k].clone() for k in ("y", "dx", "dW_gate", "dW_down", "dE_rows")}
+    for _ in range(3):
+        for k in first:
+            st.bufs[k].fill_(0)
+        st.step()
+        torch.cuda.synchronize()
+        n_u = int(st.bufs["n_unique"].item())
+        for k in first:
+            a, b = first[k], st.bufs[k]
+            if k == "dE_rows":
+                a, b = a[:n_u], b[:n_u]
+            assert torch.equal(a, b), k
+
+
+# ---------------------------------------------------------------------------------------
+# the paper-scale configurations: sampled outputs (each output row has its own definition)
+# ---------------------------------------------------------------------------------------
+def _sampled_parity(name, backward=True, n_rows=48, n_cols=40):
+    w = synth.WORKLOADS[name]
+    inp = synth.make_inputs(w)
+    st = runner.state_from_numpy(inp, B.DTYPE_BF16, w.V, backward=backward)
+    st.step(backward=backward)
+    torch.cuda.synchronize()
+    assert st.status() == B.OK
+    b = st.bufs
+    dd = O.dedup(inp["ids"])
+    n_u = int(b["n_unique"].item())
+    assert n_u == dd["n_unique"]
+    for k in ("unique_ids", "seg_offsets", "perm", "inverse"):
+        n = {"unique_ids": n_u, "seg_offsets": n_u + 1, "perm": w.T, "inverse": w.T}[k]
+        assert np.array_equal(b[k][:n].cpu().numpy(), dd[k]), k
+    rng = np.random.default_rng(1)
+    # token rows, including the first, the last and the rows around a tile edge
+    rows = np.unique(np.concatenate([[0, 127, 128, w.T - 1], rng.integers(0, w.T, n_rows)]))
+    y_ref = O.forward(inp["x"][rows], inp["ids"][rows], inp["W_gate"], inp["E"], inp["W_down"])
+    scale_y = np.abs(y_ref).max()
+    assert np.abs(_np(b["y"][rows]) - y_ref).max() / scale_y <= TOL_BF16
+    if not backward:
+        return st, inp, dd
+    bw_rows = O.backward(inp["dy"][rows], inp["x"][rows], inp["ids"][rows], inp["W_gate"], inp["E"], inp["W_down"])
+    assert O.scaled_max_err(_np(b["dx"][rows]), bw_rows["dx"]) <= TOL_BF16
+    # d_ff columns: restricting W_gate rows, E columns and W_down columns to J gives those
+    # slices of dW_gate, dW_down and dE_rows exactly
+    J = np.unique(np.concatenate([[0, 255, 256, w.d_ff - 1], rng.integers(0, w.d_ff, n_cols)]))
+    bw = O.backward(inp["dy"], inp["x"], inp["ids"], inp["W_gate"][J], inp["E"][:, J], inp["W_down"][:, J])
+    assert O.scaled_max_err(_np(b["dW_gate"][J]), bw["dW_gate"]) <= TOL_BF16
+    assert O.scaled_max_err(_np(b["dW_down"][:, J]), bw["dW_down"]) <= TOL_BF16
+    assert O.scaled_max_err(_np(b["dE_rows"][:n_u][:, J]), bw["dE_rows"]) <= TOL_BF16
+    return st, inp, dd
+
+
+def test_config_350m_sampled():
+    _sampled_parity("350m")
+
+
+def test_config_1b_sampled():
+    _sampled_parity("1b")
+
+
+def test_config_1b_long_forward_sampled():
+    st, inp, dd = _sampled_parity("1b_long_fwd", backward=False)
+    assert 9500 < dd["n_unique"] < 11000       # distinct rows grow with length
+
+
+# ---------------------------------------------------------------------------------------
+# off-device table: prefetch of the unique rows, forward/backward on the cache, write-back
+# ---------------------------------------------------------------------------------------
+def test_host_table_prefetch_and_writeback():
+    w = synth.Workload("t", 1024, 256, 512, 3000, "bf16", "zipf")
+    inp = synth.make_inputs(w, seed=80)
+    st = runner.state_from_numpy(inp, B.DTYPE_BF16, w.V)
+    st.step()
+    torch.cuda.synchronize()
+    ref = {k: st.bufs[k].clone() for k in ("y", "dx", "dW_gate", "dW_down", "dE_rows")}
+    n_u = int(st.bufs["n_unique"].item())
+
+    host_E = torch.from_numpy(inp["E"]).bfloat16().pin_memory()
+    cache = torch.zeros(min(w.T, w.V), w.d_ff, dtype=torch.bfloat16, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    B.stem_prefetch_rows(st.shape, st.bufs["unique_ids"], st.bufs["n_unique"], host_E, cache, st.bufs["ws"], side)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    expect = O.prefetch_rows(O.dedup(inp["ids"])["unique_ids"], n_u, inp["E"])
+    assert np.array_equal(cache[:n_u].float().cpu().numpy(), expect)
+    assert torch.count_nonzero(cache[n_u:]) == 0
+
+    cshape = B.make_shape(w.T, w.d_model, w.d_ff, cache.shape[0], B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    for k in ref:
+        st.bufs[k].fill_(0)
+    st.forward(ids=st.bufs["inverse"], E=cache, shape=cshape)
+    st.backward(ids=st.bufs["inverse"], E=cache, shape=cshape)
+    torch.cuda.synchronize()
+    for k in ref:
+        a, b = ref[k], st.bufs[k]
+        if k == "dE_rows":
+            a, b = a[:n_u], b[:n_u]
+        assert torch.equal(a, b), k
+
+    host_rows = torch.zeros(cache.shape[0], w.d_ff, dtype=torch.float32).pin_memory()
+    host_ids = torch.full((cache.shape[0],), -1, dtype=torch.int32).pin_memory()
+    host_n = torch.zeros(1, dtype=torch.int32).pin_memory()
+    B.stem_writeback_rows(st.shape, st.bufs["dE_rows"], st.bufs["unique_ids"], st.bufs["n_unique"], host_rows,
+                          host_ids, host_n, side)
+    side.synchronize()
+    assert int(host_n[0]) == n_u
+    assert torch.equal(host_rows[:n_u], st.bufs["dE_rows"][:n_u].cpu())
+    assert torch.equal(host_ids[:n_u], st.bufs["unique_ids"][:n_u].cpu())
+    assert torch.count_nonzero(host_rows[n_u:]) == 0
+
+    # a pageable host table is refused on the host, before any launch
+    with pytest.raises(B.StemError) as ei:
+        B.stem_prefetch_rows(st.shape, st.bufs["unique_ids"], st.bufs["n_unique"],
+                             torch.from_numpy(inp["E"]).bfloat16(), cache, st.bufs["ws"], side)
+    assert ei.value.code == B.ERR_NOT_PINNED
+    # the same call gathers from a device-resident table
+    cache.zero_()
+    B.stem_prefetch_rows(st.shape, st.bufs["unique_ids"], st.bufs["n_unique"], st.E, cache, st.bufs["ws"])
+    torch.cuda.synchronize()
+    assert np.array_equal(cache[:n_u].float().cpu().numpy(), expect)
+
+
+def test_error_paths_on_device_box():
+    w = synth.Workload("t", 64, 64, 64, 10, "bf16", "uniform")
+    inp = synth.make_inputs(w, seed=81)
+    st = runner.state_from_numpy(inp, B.DTYPE_BF16, w.V)
+    small = torch.empty(512, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.StemError) as ei:
+        B.stem_ffn_forward(st.shape, st.x, st.ids, st.W_gate, st.E, st.W_down, st.bufs["y"], None, None, small)
+    assert ei.value.code == B.ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(B.StemError) as ei:
+        B.stem_ffn_forward(st.shape, None, st.ids, st.W_gate, st.E, st.W_down, st.bufs["y"], None, None, st.bufs["ws"])
+    assert ei.value.code == B.ERR_INVALID_ARG
+    # an id outside the table is clamped and reported, the call still completes
+    st.ids[5] = 1234
+    st.forward()
+    assert st.status() == B.ERR_ID_RANGE
+    ids = inp["ids"].copy()
+    ids[5] = w.V - 1
+    y_ref = O.forward(inp["x"], ids, inp["W_gate"], inp["E"], inp["W_down"])
+    assert O.scaled_max_err(_np(st.bufs["y"]), y_ref) <= TOL_BF16
+    # T = 0 does nothing
+    z = B.make_shape(0, 64, 64, 10, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    B.stem_ffn_forward(z, None, None, None, None, None, None, None, None, st.bufs["ws"])
