@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the STEM FFN layer hot path on B200.
+
+One step = dedup of the batch's token ids + forward + backward of one layer (all steps of
+the path) on one batch of synthetic input.  Prints ONE JSON line (rank 0).
+
+    python bench.py --gpus 1 --steps 30 --warmup 5
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference ...        # the CPU checker, timed on the host cores
+
+N > 1 runs N independent replicas (the path has no exchange step): every rank processes
+its own batch, no data-path collective; the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2601_10639_b200 import synth  # noqa: E402
+
+METRIC = "STEM-FFN fwd+bwd tokens/sec (1B-class layer, dedup + forward + backward)"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+def load_traffic(workload: str):
+    p = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f).get(workload, {})
+    return {}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def __exit__(self, *exc):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float) -> dict:
+        sm, mx, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.2] or [l for (_, l) in self.lines]
+        for line in rows:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": max(mx), "power_w_max": max(power),
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_tokens_per_sec(inputs: dict, Tc: int) -> tuple[float, float]:
+    """Time the CPU checker (as it stands) on the first Tc tokens of the batch."""
+    from oracle import stem_oracle as O
+    sl = {k: (v[:Tc] if k in ("x", "dy", "ids") else v) for k, v in inputs.items()}
+    t = time.perf_counter()
+    O.dedup(sl["ids"])
+    O.forward(sl["x"], sl["ids"], sl["W_gate"], sl["E"], sl["W_down"])
+    O.backward(sl["dy"], sl["x"], sl["ids"], sl["W_gate"], sl["E"], sl["W_down"])
+    dt = time.perf_counter() - t
+    return Tc / dt, dt
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, w):
+    """The CPU checker as the reference arm: rank 0 only, bounded token sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    Tc = args.ref_tokens
+    inputs = synth.make_inputs(w, T=Tc)
+    for _ in range(args.warmup):
+        oracle_tokens_per_sec(inputs, Tc)
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_tokens_per_sec(inputs, Tc)
+    dt = time.perf_counter() - t
+    value = Tc * args.steps / dt
+    sample = f"first {Tc} tokens of the batch per step (every stage is linear in T), all weights and the full table"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "T": w.T, "d_model": w.d_model, "d_ff": w.d_ff, "V": w.V, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="stem", choices=["stem", "reference"])
+    ap.add_argument("--workload", default="1b", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--cpu-tokens", type=int, default=8192, help="tokens in the CPU-baseline sample (0 = skip)")
+    ap.add_argument("--ref-tokens", type=int, default=1024, help="tokens per step of --impl reference")
+    ap.add_argument("--seed", type=int, default=synth.BASE_SEED)
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.warmup < 3:
+        args.warmup = 3
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2601_10639_b200 import binding as B
+    from paper_2601_10639_b200 import runner
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()  # fail loudly here if the extension is missing
+
+    dcode = B.DTYPE_BF16 if w.dtype == "bf16" else B.DTYPE_FP32
+    dt = runner.torch_dtype(dcode)
+    T, d, F, V = w.T, w.d_model, w.d_ff, w.V
+    backward = w.backward
+    # ---- synthetic inputs (every rank its own batch; same shapes) -----------------------
+    gen = torch.Generator(device=dev).manual_seed(args.seed + 1000 * rank)
+    st = runner.LayerState(B.make_shape(T, d, F, V, dcode, B.DTYPE_FP32, 0), device=dev)
+    st.x = torch.randn(T, d, generator=gen, device=dev, dtype=torch.float32).to(dt)
+    st.dy = torch.randn(T, d, generator=gen, device=dev, dtype=torch.float32).to(dt)
+    st.W_gate = (torch.randn(F, d, generator=gen, device=dev, dtype=torch.float32) * d ** -0.5).to(dt)
+    st.W_down = (torch.randn(d, F, generator=gen, device=dev, dtype=torch.float32) * F ** -0.5).to(dt)
+    st.E = torch.empty(V, F, device=dev, dtype=dt)
+    for r0 in range(0, V, 4096):
+        r1 = min(V, r0 + 4096)
+        st.E[r0:r1] = (torch.randn(r1 - r0, F, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(dt)
+    ids_np = synth.token_ids(args.seed + rank, T, V, w.id_dist)
+    st.ids = torch.from_numpy(ids_np).to(dev)
+    st.allocate(backward)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ------------------------------------------------------------
+    for _ in range(args.warmup):
+        st.step(backward=backward)
+    barrier()
+    assert st.status() == B.OK, B.status_string(st.status())
+    n_u = int(st.bufs["n_unique"].item())
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = B.stem_launch_count()
+    with ClockSampler(local) as clocks:
+        B.stem_profile_enable(True)
+        barrier()
+        t0 = time.time()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            st.step(backward=backward)
+        ev1.record(stream)
+        barrier()
+        t1 = time.time()
+        B.stem_profile_enable(False)
+    launches = B.stem_launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    records = B.stem_profile_records()
+    assert st.status() == B.OK, B.status_string(st.status())
+    clock_summary = clocks.summary(t0, t1)
+
+    # ---- end to end through the host-buffer entry point -------------------------------------
+    esz = 2 if dcode == B.DTYPE_BF16 else 4
+    e2e = None
+    if backward:
+        hx, hdy = st.x.cpu().pin_memory(), st.dy.cpu().pin_memory()
+        hids = st.ids.cpu().pin_memory()
+        hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+        hn = torch.zeros(1, dtype=torch.int32).pin_memory()
+        arena = torch.empty(B.stem_step_arena_bytes(st.shape), dtype=torch.uint8, device=dev)
+        B.stem_init_workspace(arena)
+        b = st.bufs
+
+        def host_step():
+            B.stem_ffn_step_host(st.shape, hx, hids, hdy, st.W_gate, st.E, st.W_down, hy, hdx, b["dW_gate"],
+                                 b["dW_down"], b["dE_rows"], b["unique_ids"], b["n_unique"], hn, arena)
+        for _ in range(3):
+            host_step()
+        barrier()
+        ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ee0.record(stream)
+        for _ in range(args.steps):
+            host_step()
+        ee1.record(stream)
+        barrier()
+        e2e_ms = ee0.elapsed_time(ee1)
+        assert B.stem_query_status(arena) == B.OK
+        assert int(hn[0]) == n_u
+        assert torch.equal(hy, st.bufs["y"].cpu())       # same result as the device-resident path
+        e2e = {"ms": e2e_ms, "h2d": 2 * T * d * esz + T * 4, "d2h": 2 * T * d * esz + 4}
+        del arena
+
+    # ---- max over ranks ------------------------------------------------------------------------
+    if world > 1:
+        t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t[0])
+        if e2e:
+            e2e["ms"] = float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    ms_per_step = ms_total / args.steps
+    value = world * T * args.steps / (ms_total * 1e-3)
+
+    # ---- per-kernel figures ------------------------------------------------------------------------
+    by_name: dict[str, list] = {}
+    for name, ms in records:
+        by_name.setdefault(name, []).append(ms)
+    flops_gemm = 2.0 * T * d * F
+    gbytes = 4 if st.shape.grad_dtype == B.DTYPE_FP32 else 2
+    seg_bytes = T * F * esz + n_u * F * gbytes + 4 * (T + n_u + 1)
+    kernels = {}
+    for name, v in by_name.items():
+        avg = float(np.mean(v))
+        k = {"launch_sets": len(v), "avg_ms": avg, "share": float(np.sum(v)) / ms_total}
+        if name.endswith("_gemm"):
+            k["tflops"] = flops_gemm / (avg * 1e-3) / 1e12
+            k["frac_of_measured_sustained"] = k["tflops"] / peaks["bf16_tflops_sustained"]
+            k["frac_of_measured_burst"] = k["tflops"] / peaks["bf16_tflops"]
+        elif name == "seg_reduce":
+            k["gbs"] = seg_bytes / (avg * 1e-3) / 1e9
+            k["frac_of_measured_hbm"] = k["gbs"] / peaks["hbm_gbs"]
+        kernels[name] = k
+    gemms = {n: k for n, k in kernels.items() if n.endswith("_gemm")}
+    traffic = load_traffic(w.name)
+    roofline = None
+    if gemms and dcode == B.DTYPE_BF16:
+        dom = max(gemms, key=lambda n: gemms[n]["avg_ms"])
+        roofline = {"kernel": dom, "bound": "tensor", "achieved": gemms[dom]["tflops"],
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "frac": gemms[dom]["tflops"] / peaks["bf16_tflops_sustained"],
+                    "traffic": traffic.get(dom), "peak_source": peaks["source"] + " (sustained bf16 GEMM)",
+                    "flops_per_launch": flops_gemm}
+
+    # ---- the CPU checker timed beside it (rank 0, N = 1 only) -----------------------------------------
+    cpu = None
+    if world == 1 and args.cpu_tokens > 0 and backward:
+        Tc = min(args.cpu_tokens, T)
+        host_inputs = {"x": st.x[:Tc].float().cpu().numpy(), "dy": st.dy[:Tc].float().cpu().numpy(),
+                       "ids": ids_np[:Tc], "W_gate": st.W_gate.float().cpu().numpy(),
+                       "W_down": st.W_down.float().cpu().numpy(), "E": st.E.float().cpu().numpy()}
+        tps, secs = oracle_tokens_per_sec(host_inputs, Tc)
+        cpu = {"value": tps, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle", "seconds": secs,
+               "sample": f"first {Tc} of {T} tokens, full weights and table, dedup + forward + backward in fp64"}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if dcode == B.DTYPE_BF16 else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "T": T, "d_model": d, "d_ff": F, "V": V, "ids": w.id_dist,
+                   "n_unique": n_u, "backward": backward, "parallelism": f"replicas x{world}",
+                   "l2": "per-step working set (~2.5 GB at 1b shapes) exceeds the 126 MB L2; no flush"},
+        "gpu_launches": int(launches),
+        "tflops_step": (12.0 if backward else 4.0) * T * d * F / (ms_per_step * 1e-3) / 1e12,
+        "clocks": clock_summary,
+        "roofline": roofline,
+        "kernels": kernels,
+        "cpu_baseline": cpu,
+    }
+    if e2e:
+        out["e2e"] = {"value": world * T * args.steps / (e2e["ms"] * 1e-3), "unit": "tokens/s",
+                      "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                      "ms_per_step": e2e["ms"] / args.steps}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

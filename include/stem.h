@@ -164,11 +164,47 @@ int stem_writeback_rows(const stem_shape_t* shape, const void* dE_rows, const in
  * step is exactly this; exposed for testing and reuse):
  *   C[m,n] = sum_k A(m,k) B(n,k),  C row-major [M,N] (bf16 if c_fp32 == 0, else fp32).
  * a_mn == 0: A stored [M,K] row-major (K contiguous); a_mn == 1: A stored [K,M]
- * row-major (M contiguous).  b_mn likewise for B ([N,K] or [K,N]).  M, N, K multiples
- * of 8.  bf16 inputs, fp32 accumulation.  ws: a workspace (status word only).
+ * row-major (M contiguous).  b_mn likewise for B ([N,K] or [K,N]).  N and the contiguous
+ * extent of each operand must be multiples of 8.  bf16 inputs, fp32 accumulation.
+ * ws: a workspace (status word only).
  */
 int stem_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t a_mn, const void* B,
                    int32_t b_mn, void* C, int32_t c_fp32, int32_t flags, void* ws, void* stream);
+
+/*
+ * One training step of the layer from host buffers (the composition of the calls above,
+ * in the order Section 3.3 gives for training: ids deduplicated, forward, backward, table
+ * gradients reduced per unique id):
+ *   copy host_x, host_ids, host_dy to the device; stem_dedup_ids; stem_ffn_forward;
+ *   stem_ffn_backward; copy y and dx back to host_y, host_dx (and n_u to host_n_unique
+ *   when it is not NULL).
+ * host_*: host memory ([T,d_model] in dtype; ids [T] int32), page-locked for the copies
+ * to be asynchronous.  W_gate, E, W_down: device-resident parameters.  dW_gate, dW_down,
+ * dE_rows, unique_ids [min(T,V)], n_unique [1]: device outputs, as in stem_ffn_backward
+ * (they stay on the device for the optimizer).  arena: device scratch of
+ * stem_step_arena_bytes() bytes holding the workspace (call stem_init_workspace on it
+ * once) and every intermediate.  Everything is enqueued on `stream`.
+ */
+int stem_step_arena_bytes(const stem_shape_t* shape, size_t* bytes /*host, out*/);
+int stem_ffn_step_host(const stem_shape_t* shape, const void* host_x, const int32_t* host_ids,
+                       const void* host_dy, const void* W_gate, const void* E, const void* W_down,
+                       void* host_y, void* host_dx, void* dW_gate, void* dW_down, void* dE_rows,
+                       int32_t* unique_ids, int32_t* n_unique, int32_t* host_n_unique /*host*/,
+                       void* arena, size_t arena_bytes, void* stream);
+
+/*
+ * Instrumentation (no counterpart in the paper).  stem_launch_count: kernels this library
+ * has launched in this process.  stem_profile_enable(1) clears earlier records and starts
+ * recording one CUDA-event pair per step of the path (dedup, gate_gemm, down_gemm,
+ * dh_gemm, dw_down_gemm, seg_reduce, dw_gate_gemm, dx_gemm, prefetch_rows,
+ * writeback_rows, h2d_inputs, d2h_outputs) on the stream of each call; (0) stops.
+ * stem_profile_get waits for record i to finish and returns its name (static storage) and
+ * its duration in milliseconds.
+ */
+long long stem_launch_count(void);
+int stem_profile_enable(int on);
+int stem_profile_count(void);
+int stem_profile_get(int i, const char** name /*host, out*/, float* ms /*host, out*/);
 
 #ifdef __cplusplus
 }

@@ -26,7 +26,8 @@ FLAG_SIMT = 1
 EXPORTS = (
     "stem_version", "stem_status_string", "stem_workspace_bytes", "stem_init_workspace",
     "stem_query_status", "stem_dedup_ids", "stem_ffn_forward", "stem_ffn_backward",
-    "stem_prefetch_rows", "stem_writeback_rows", "stem_gemm_bf16",
+    "stem_prefetch_rows", "stem_writeback_rows", "stem_gemm_bf16", "stem_step_arena_bytes",
+    "stem_ffn_step_host", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
 )
 
 
@@ -67,7 +68,14 @@ def lib() -> ctypes.CDLL:
             "stem_prefetch_rows": [shp, vp, vp, vp, vp, vp, vp],
             "stem_writeback_rows": [shp, vp, vp, vp, vp, vp, vp, vp],
             "stem_gemm_bf16": [i32, i32, i32, vp, i32, vp, i32, vp, i32, i32, vp, vp],
+            "stem_step_arena_bytes": [shp, ctypes.POINTER(sz)],
+            "stem_ffn_step_host": [shp] + [vp] * 15 + [sz, vp],
+            "stem_profile_enable": [ctypes.c_int],
+            "stem_profile_count": [],
+            "stem_profile_get": [ctypes.c_int, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float)],
         }
+        L.stem_launch_count.restype = ctypes.c_longlong
+        L.stem_launch_count.argtypes = []
         for name, args in sigs.items():
             fn = getattr(L, name)
             fn.restype = ctypes.c_int
@@ -159,3 +167,35 @@ def stem_writeback_rows(shape, dE_rows, unique_ids, n_rows, host_rows, host_ids,
 def stem_gemm_bf16(M, N, K, A, a_mn, B, b_mn, C, c_fp32, flags, ws, stream=None) -> None:
     _check(lib().stem_gemm_bf16(M, N, K, _p(A), int(a_mn), _p(B), int(b_mn), _p(C), int(c_fp32), flags, _p(ws),
                                 _stream(stream)), "stem_gemm_bf16")
+
+
+def stem_step_arena_bytes(shape: StemShape) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().stem_step_arena_bytes(ctypes.byref(shape), ctypes.byref(out)), "stem_step_arena_bytes")
+    return out.value
+
+
+def stem_ffn_step_host(shape, host_x, host_ids, host_dy, W_gate, E, W_down, host_y, host_dx, dW_gate, dW_down,
+                       dE_rows, unique_ids, n_unique, host_n_unique, arena, stream=None) -> None:
+    _check(lib().stem_ffn_step_host(ctypes.byref(shape), _p(host_x), _p(host_ids), _p(host_dy), _p(W_gate), _p(E),
+                                    _p(W_down), _p(host_y), _p(host_dx), _p(dW_gate), _p(dW_down), _p(dE_rows),
+                                    _p(unique_ids), _p(n_unique), _p(host_n_unique), _p(arena),
+                                    arena.numel() * arena.element_size(), _stream(stream)), "stem_ffn_step_host")
+
+
+def stem_launch_count() -> int:
+    return lib().stem_launch_count()
+
+
+def stem_profile_enable(on: bool) -> None:
+    _check(lib().stem_profile_enable(1 if on else 0), "stem_profile_enable")
+
+
+def stem_profile_records() -> list:
+    """[(name, milliseconds), ...] for every record since stem_profile_enable(True)."""
+    out = []
+    name, ms = ctypes.c_char_p(), ctypes.c_float()
+    for i in range(lib().stem_profile_count()):
+        _check(lib().stem_profile_get(i, ctypes.byref(name), ctypes.byref(ms)), "stem_profile_get")
+        out.append((name.value.decode(), ms.value))
+    return out

@@ -1,6 +1,9 @@
 // C ABI of libstem: argument checks, workspace carve-up and kernel sequencing.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "stem_internal.h"
 
@@ -19,8 +22,45 @@ int device_sm_count() {
 }
 
 namespace {
+std::atomic<long long> g_launches{0};
+}
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+namespace {
 
 thread_local char g_cuda_msg[256] = "";
+
+// Optional per-step timing: a pair of CUDA events around each step of the path, recorded
+// on the caller's stream.  Off by default; a few microseconds per step when on.
+struct ProfRecord { const char* name; cudaEvent_t begin, end; };
+std::mutex g_prof_mutex;
+bool g_prof_on = false;
+std::vector<ProfRecord> g_prof;        // records of the current session
+std::vector<cudaEvent_t> g_event_pool;  // events kept for reuse
+
+cudaEvent_t take_event() {
+  if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+struct ProfScope {
+  cudaStream_t st; int idx = -1;
+  ProfScope(const char* name, cudaStream_t s) : st(s) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    if (!g_prof_on) return;
+    ProfRecord r{name, take_event(), take_event()};
+    cudaEventRecord(r.begin, st);
+    g_prof.push_back(r);
+    idx = static_cast<int>(g_prof.size()) - 1;
+  }
+  ~ProfScope() {
+    if (idx < 0) return;
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    if (idx < static_cast<int>(g_prof.size())) cudaEventRecord(g_prof[idx].end, st);
+  }
+};
 
 int cuda_fail(cudaError_t e) {
   snprintf(g_cuda_msg, sizeof(g_cuda_msg), "CUDA error: %s", cudaGetErrorString(e));
@@ -155,6 +195,7 @@ int stem_dedup_ids(const stem_shape_t* shape, const int32_t* ids, int32_t* uniqu
   if (shape->T > 0 && !ids) return STEM_ERR_INVALID_ARG;
   const WsLayout w = ws_layout(shape);
   if (ws_bytes < w.total) return STEM_ERR_WORKSPACE_TOO_SMALL;
+  ProfScope prof("dedup", static_cast<cudaStream_t>(stream));
   cudaError_t e = launch_dedup(shape->T, shape->V, ids, unique_ids, n_unique, inverse, perm, seg_offsets,
                                static_cast<char*>(ws) + w.dedup_off, status_of(ws), static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
@@ -179,11 +220,18 @@ int stem_ffn_forward(const stem_shape_t* shape, const void* x, const int32_t* id
 
   EpiParams gate;
   gate.ids = ids; gate.E = E; gate.V = shape->V; gate.H = H; gate.G = G_save; gate.status = status_of(ws);
-  cudaError_t e = gemm(shape, T, F, d, x, false, W_gate, false, kEpiGate, gate, st);   // G = x W_gate^T, fused lookup
+  cudaError_t e;
+  {
+    ProfScope prof("gate_gemm", st);
+    e = gemm(shape, T, F, d, x, false, W_gate, false, kEpiGate, gate, st);   // G = x W_gate^T, fused lookup
+  }
   if (e != cudaSuccess) return cuda_fail(e);
   EpiParams down;
   down.out = y; down.out_fp32 = shape->dtype == STEM_DTYPE_FP32; down.status = status_of(ws);
-  e = gemm(shape, T, d, F, H, false, W_down, false, kEpiStore, down, st);              // y = H W_down^T
+  {
+    ProfScope prof("down_gemm", st);
+    e = gemm(shape, T, d, F, H, false, W_down, false, kEpiStore, down, st);              // y = H W_down^T
+  }
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
 }
 
@@ -217,25 +265,33 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
   // dU = dH SiLU(G), dG = dH E[ids] SiLU'(G)
   EpiParams dh;
   dh.ids = ids; dh.E = E; dh.V = shape->V; dh.H = dU; dh.G = dG; dh.Gin = G_save; dh.status = status_of(ws);
-  cudaError_t e = gemm(shape, T, F, d, dy, false, W_down, true, kEpiDH, dh, st);
+  cudaError_t e;
+  {
+    ProfScope prof("dh_gemm", st);
+    e = gemm(shape, T, F, d, dy, false, W_down, true, kEpiDH, dh, st);
+  }
   if (e != cudaSuccess) return cuda_fail(e);
   if (dW_down) {  // dW_down[i,j] = sum_t dy[t,i] H[t,j]
     EpiParams p; p.out = dW_down; p.out_fp32 = grad_fp32; p.status = status_of(ws);
+    ProfScope prof("dw_down_gemm", st);
     e = gemm(shape, d, F, T, dy, true, H_save, true, kEpiStore, p, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
   if (dE_rows) {
+    ProfScope prof("seg_reduce", st);
     e = launch_segreduce(T, F, shape->dtype, shape->grad_dtype, dU, perm, seg_offsets, n_unique, dE_rows,
                          base + w.part_off, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
   if (dW_gate) {  // dW_gate[j,k] = sum_t dG[t,j] x[t,k]
     EpiParams p; p.out = dW_gate; p.out_fp32 = grad_fp32; p.status = status_of(ws);
+    ProfScope prof("dw_gate_gemm", st);
     e = gemm(shape, F, d, T, dG, true, x, true, kEpiStore, p, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
   if (dx) {  // dx = dG W_gate (contraction over d_ff; W_gate is [F, d]: d contiguous)
     EpiParams p; p.out = dx; p.out_fp32 = shape->dtype == STEM_DTYPE_FP32; p.status = status_of(ws);
+    ProfScope prof("dx_gemm", st);
     e = gemm(shape, T, d, F, dG, false, W_gate, true, kEpiStore, p, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
@@ -251,6 +307,7 @@ int stem_prefetch_rows(const stem_shape_t* shape, const int32_t* ids, const int3
   if (int rc = pinned_or_device(table, &src)) return rc;
   const int max_rows = shape->T < shape->V ? shape->T : shape->V;
   const size_t row_bytes = static_cast<size_t>(shape->d_ff) * elem_bytes(shape->dtype);
+  ProfScope prof("prefetch_rows", static_cast<cudaStream_t>(stream));
   cudaError_t e = launch_gather_rows(max_rows, shape->V, row_bytes, ids, n_ids, src, dev_cache,
                                      ws ? status_of(ws) : nullptr, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
@@ -270,6 +327,7 @@ int stem_writeback_rows(const stem_shape_t* shape, const void* dE_rows, const in
   if (int rc = pinned_or_device(host_n, &hn)) return rc;
   const int max_rows = shape->T < shape->V ? shape->T : shape->V;
   const size_t row_bytes = static_cast<size_t>(shape->d_ff) * elem_bytes(shape->grad_dtype);
+  ProfScope prof("writeback_rows", static_cast<cudaStream_t>(stream));
   cudaError_t e = launch_writeback_rows(max_rows, row_bytes, dE_rows, unique_ids, n_rows, const_cast<void*>(hr),
                                         static_cast<int32_t*>(const_cast<void*>(hi)),
                                         static_cast<int32_t*>(const_cast<void*>(hn)), static_cast<cudaStream_t>(stream));
@@ -281,7 +339,7 @@ int stem_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t a_mn,
   if (M < 0 || N < 0 || K <= 0) return STEM_ERR_INVALID_ARG;
   if (M == 0 || N == 0) return STEM_OK;
   if (!A || !B || !C || !ws || !aligned16(A) || !aligned16(B) || !aligned16(C)) return STEM_ERR_INVALID_ARG;
-  if ((M % 8) || (N % 8) || (K % 8)) return STEM_ERR_UNSUPPORTED_SHAPE;
+  if ((N % 8) || ((a_mn ? M : K) % 8) || ((b_mn ? N : K) % 8)) return STEM_ERR_UNSUPPORTED_SHAPE;
   EpiParams p; p.out = C; p.out_fp32 = c_fp32; p.status = status_of(ws);
   cudaError_t e;
   if (flags & STEM_FLAG_SIMT) {
@@ -289,6 +347,100 @@ int stem_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t a_mn,
   } else {
     if (!is_sm100()) return STEM_ERR_UNSUPPORTED_ARCH;
     e = launch_tc_gemm(M, N, K, A, a_mn != 0, B, b_mn != 0, kEpiStore, p, static_cast<cudaStream_t>(stream));
+  }
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
+long long stem_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int stem_profile_enable(int on) {
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  if (on) {
+    for (const ProfRecord& r : g_prof) { g_event_pool.push_back(r.begin); g_event_pool.push_back(r.end); }
+    g_prof.clear();
+  }
+  g_prof_on = on != 0;
+  return STEM_OK;
+}
+
+int stem_profile_count(void) {
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  return static_cast<int>(g_prof.size());
+}
+
+int stem_profile_get(int i, const char** name, float* ms) {
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  if (i < 0 || i >= static_cast<int>(g_prof.size()) || !name || !ms) return STEM_ERR_INVALID_ARG;
+  cudaError_t e = cudaEventSynchronize(g_prof[i].end);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(ms, g_prof[i].begin, g_prof[i].end);
+  if (e != cudaSuccess) return cuda_fail(e);
+  *name = g_prof[i].name;
+  return STEM_OK;
+}
+
+namespace {
+struct Arena {
+  size_t ws, ws_bytes, x, dy, ids, y, dx, G, H, inverse, perm, seg, total;
+};
+Arena arena_layout(const stem_shape_t* s) {
+  Arena a{};
+  const size_t T = s->T, td = align_up(T * s->d_model * elem_bytes(s->dtype), 256),
+               tf = align_up(T * s->d_ff * elem_bytes(s->dtype), 256), ti = align_up((T + 1) * 4, 256);
+  const size_t R = static_cast<size_t>(s->T < s->V ? s->T : s->V);
+  size_t o = 0;
+  a.ws = o; a.ws_bytes = ws_layout(s).total; o += a.ws_bytes;
+  a.x = o; o += td;  a.dy = o; o += td;  a.ids = o; o += ti;
+  a.y = o; o += td;  a.dx = o; o += td;  a.G = o; o += tf;  a.H = o; o += tf;
+  a.inverse = o; o += ti;  a.perm = o; o += ti;  a.seg = o; o += align_up((R + 1) * 4, 256);
+  a.total = o;
+  return a;
+}
+}  // namespace
+
+int stem_step_arena_bytes(const stem_shape_t* shape, size_t* bytes) {
+  if (!bytes) return STEM_ERR_INVALID_ARG;
+  if (int rc = check_shape(shape)) return rc;
+  *bytes = arena_layout(shape).total;
+  return STEM_OK;
+}
+
+int stem_ffn_step_host(const stem_shape_t* shape, const void* host_x, const int32_t* host_ids, const void* host_dy,
+                       const void* W_gate, const void* E, const void* W_down, void* host_y, void* host_dx,
+                       void* dW_gate, void* dW_down, void* dE_rows, int32_t* unique_ids, int32_t* n_unique,
+                       int32_t* host_n_unique, void* arena, size_t arena_bytes, void* stream) {
+  if (int rc = check_shape(shape)) return rc;
+  if (!arena || !aligned16(arena)) return STEM_ERR_INVALID_ARG;
+  if (shape->T == 0) return STEM_OK;
+  if (!host_x || !host_ids || !host_dy || !host_y || !host_dx || !unique_ids || !n_unique) return STEM_ERR_INVALID_ARG;
+  const Arena a = arena_layout(shape);
+  if (arena_bytes < a.total) return STEM_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = static_cast<char*>(arena);
+  const size_t td = static_cast<size_t>(shape->T) * shape->d_model * elem_bytes(shape->dtype);
+  cudaError_t e;
+  {
+    ProfScope prof("h2d_inputs", st);
+    e = cudaMemcpyAsync(base + a.ids, host_ids, static_cast<size_t>(shape->T) * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(base + a.x, host_x, td, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(base + a.dy, host_dy, td, cudaMemcpyHostToDevice, st);
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+  int32_t* ids = reinterpret_cast<int32_t*>(base + a.ids);
+  int32_t* perm = reinterpret_cast<int32_t*>(base + a.perm);
+  int32_t* seg = reinterpret_cast<int32_t*>(base + a.seg);
+  if (int rc = stem_dedup_ids(shape, ids, unique_ids, n_unique, reinterpret_cast<int32_t*>(base + a.inverse), perm, seg,
+                              base + a.ws, a.ws_bytes, stream)) return rc;
+  if (int rc = stem_ffn_forward(shape, base + a.x, ids, W_gate, E, W_down, base + a.y, base + a.G, base + a.H,
+                                base + a.ws, a.ws_bytes, stream)) return rc;
+  if (int rc = stem_ffn_backward(shape, base + a.dy, base + a.x, ids, W_gate, E, W_down, base + a.G, base + a.H, perm,
+                                 seg, n_unique, base + a.dx, dW_gate, dW_down, dE_rows, unique_ids, base + a.ws,
+                                 a.ws_bytes, stream)) return rc;
+  {
+    ProfScope prof("d2h_outputs", st);
+    e = cudaMemcpyAsync(host_y, base + a.y, td, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(host_dx, base + a.dx, td, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && host_n_unique)
+      e = cudaMemcpyAsync(host_n_unique, n_unique, 4, cudaMemcpyDeviceToHost, st);
   }
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
 }

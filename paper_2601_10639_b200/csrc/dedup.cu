@@ -189,6 +189,7 @@ cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, 
                          int32_t* status, cudaStream_t stream) {
   if (T <= 0) {
     empty_dedup_kernel<<<1, 1, 0, stream>>>(n_unique, seg_offsets);
+    count_launches(1);
     return cudaGetLastError();
   }
   const int epw = elems_per_warp(T);
@@ -212,10 +213,12 @@ cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, 
     scan_exclusive_kernel<<<1, 1024, 0, stream>>>(counts, n_warps * kRadix);
     radix_scatter_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(T, V, epw, n_warps, pass * 8, first,
                                                                     kin, vin, counts, kout, vout);
+    count_launches(3);
     kin = kout;
     vin = vout;
   }
   segment_heads_kernel<<<1, 1024, 0, stream>>>(T, kin, perm, unique_ids, n_unique, inverse, seg_offsets);
+  count_launches(1);
   return cudaGetLastError();
 }
 

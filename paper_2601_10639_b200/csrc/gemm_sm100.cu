@@ -349,6 +349,7 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, int M, i
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = tiles < device_sm_count() ? tiles : device_sm_count();
   kern<<<grid, kThreads, L::kTotal, stream>>>(tmA, tmB, M, N, K, 8, ep);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -368,7 +369,9 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
 cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const void* B, bool b_mn,
                            EpiKind kind, const EpiParams& ep, cudaStream_t stream) {
   if (M <= 0 || N <= 0) return cudaSuccess;
-  if (K <= 0 || (M % 8) || (N % 8) || (K % 8)) return cudaErrorNotSupported;
+  // TMA needs 16-byte row pitches (the contiguous extent of each operand a multiple of 8
+  // elements); the epilogue stores 8 columns at a time.
+  if (K <= 0 || (N % 8) || ((a_mn ? M : K) % 8) || ((b_mn ? N : K) % 8)) return cudaErrorNotSupported;
   // layer call sites: gate (K,K,gate)  down (K,K,store)  dH (K,MN,dh)  dx (K,MN,store)
   //                   dW_down / dW_gate (MN,MN,store); the plain-GEMM entry adds (MN,K,store)
   if (!a_mn && !b_mn) {

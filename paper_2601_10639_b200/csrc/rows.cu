@@ -68,6 +68,7 @@ cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int3
   if (blocks > cap) blocks = cap;
   gather_rows_kernel<<<blocks, kThreads, 0, stream>>>(V, vec, ids, n_ids, static_cast<const uint4*>(table),
                                                      static_cast<uint4*>(dst), status);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -79,6 +80,7 @@ cudaError_t launch_writeback_rows(int max_rows, size_t row_bytes, const void* ro
   const int blocks = device_sm_count() * 4;
   writeback_rows_kernel<<<blocks, kThreads, 0, stream>>>(vec, static_cast<const uint4*>(rows), unique_ids,
                                                         n_rows, static_cast<uint4*>(host_rows), host_ids, host_n);
+  count_launches(1);
   return cudaGetLastError();
 }
 

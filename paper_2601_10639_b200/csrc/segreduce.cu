@@ -188,6 +188,7 @@ cudaError_t launch_typed(int T, int F, const void* dU, const int32_t* perm, cons
       static_cast<float*>(scratch));
   segreduce_pass2_kernel<TOut, VI><<<grid, kThreads, 0, stream>>>(
       T, F, seg_offsets, n_unique, static_cast<const float*>(scratch), static_cast<TOut*>(dE_rows));
+  count_launches(2);
   return cudaGetLastError();
 }
 

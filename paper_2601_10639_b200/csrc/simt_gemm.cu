@@ -115,6 +115,7 @@ cudaError_t launch_kind(int M, int N, int K, const void* A, const void* B, EpiKi
     case kEpiGate: simt_gemm_kernel<T, A_MN, B_MN, kEpiGate><<<grid, 256, 0, stream>>>(M, N, K, a, b, ep); break;
     case kEpiDH: simt_gemm_kernel<T, A_MN, B_MN, kEpiDH><<<grid, 256, 0, stream>>>(M, N, K, a, b, ep); break;
   }
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -87,5 +87,6 @@ cudaError_t launch_writeback_rows(int max_rows, size_t row_bytes, const void* ro
                                   int32_t* host_ids, int32_t* host_n, cudaStream_t stream);
 
 int device_sm_count();
+void count_launches(int n);  // bookkeeping for stem_launch_count()
 
 }  // namespace stem
