@@ -49,6 +49,7 @@ extern "C" {
 #define STEM_ERR_CUDA (-6)
 #define STEM_ERR_TIMEOUT (-7)  /* device: a bounded pipeline wait expired          */
 #define STEM_ERR_ID_RANGE (-8) /* device: a token id was outside [0,V) (clamped)  */
+#define STEM_ERR_STATIC_LIMIT (-9) /* size beyond the fixed scratch of an allocation-free call */
 
 #define STEM_DTYPE_FP32 0
 #define STEM_DTYPE_BF16 1
@@ -99,6 +100,31 @@ int stem_query_status(const void* ws, void* stream, int32_t* status_out /*host*/
 int stem_dedup_ids(const stem_shape_t* shape, const int32_t* ids, int32_t* unique_ids,
                    int32_t* n_unique, int32_t* inverse, int32_t* perm, int32_t* seg_offsets,
                    void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * stem_dedup_ids for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a deployment aid).  Think of an inference server whose framework
+ * claimed all of HBM for weights and KV cache at start-up, a plug-in invoked from inside
+ * another runtime that forbids allocation on its threads, or a latency-critical loop in
+ * which a cudaMalloc would stall every stream of the device: none of them can produce
+ * the workspace stem_dedup_ids wants.  Here the sort's scratch is a fixed 1.25 MiB array
+ * compiled into the library (held by every GPU that loads it, until the process exits),
+ * so the call takes inputs and outputs only and calls no allocator of any kind.
+ *   - Same outputs, bit for bit, as stem_dedup_ids.  Only shape->T and shape->V are read.
+ *   - Limit: T <= stem_dedup_static_max_tokens() (65536); larger T returns
+ *     STEM_ERR_STATIC_LIMIT and launches nothing.
+ *   - status: optional device int32[4], zeroed by the caller; receives STEM_ERR_ID_RANGE
+ *     if an id is outside [0,V) (ids are clamped either way).  NULL = not reported.
+ *   - The first call on each device looks up the array's device address; make that first
+ *     call before starting any stream capture on that device.
+ *   - All calls on a device share the one array: two calls whose kernels can overlap on
+ *     the GPU (different streams, no ordering between them) race.  Order them.  The array
+ *     keeps the previous call's contents; nothing in it needs clearing between calls.
+ */
+int stem_dedup_ids_static(const stem_shape_t* shape, const int32_t* ids, int32_t* unique_ids,
+                          int32_t* n_unique, int32_t* inverse, int32_t* perm, int32_t* seg_offsets,
+                          int32_t* status, void* stream);
+int stem_dedup_static_max_tokens(void);
 
 /*
  * Forward (Section 3.1, the layer equation).  Two kernels:

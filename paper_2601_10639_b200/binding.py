@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libstem.so")
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_ARCH = -1, -2, -3
 ERR_WORKSPACE_TOO_SMALL, ERR_NOT_PINNED, ERR_CUDA, ERR_TIMEOUT, ERR_ID_RANGE = -4, -5, -6, -7, -8
+ERR_STATIC_LIMIT = -9
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 FLAG_SIMT = 1
 
@@ -28,6 +29,7 @@ EXPORTS = (
     "stem_query_status", "stem_dedup_ids", "stem_ffn_forward", "stem_ffn_backward",
     "stem_prefetch_rows", "stem_writeback_rows", "stem_gemm_bf16", "stem_step_arena_bytes",
     "stem_ffn_step_host", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
+    "stem_dedup_ids_static", "stem_dedup_static_max_tokens",
 )
 
 
@@ -69,6 +71,8 @@ def lib() -> ctypes.CDLL:
             "stem_writeback_rows": [shp, vp, vp, vp, vp, vp, vp, vp],
             "stem_gemm_bf16": [i32, i32, i32, vp, i32, vp, i32, vp, i32, i32, vp, vp],
             "stem_step_arena_bytes": [shp, ctypes.POINTER(sz)],
+            "stem_dedup_ids_static": [shp, vp, vp, vp, vp, vp, vp, vp, vp],
+            "stem_dedup_static_max_tokens": [],
             "stem_ffn_step_host": [shp] + [vp] * 15 + [sz, vp],
             "stem_profile_enable": [ctypes.c_int],
             "stem_profile_count": [],
@@ -199,3 +203,14 @@ def stem_profile_records() -> list:
         _check(lib().stem_profile_get(i, ctypes.byref(name), ctypes.byref(ms)), "stem_profile_get")
         out.append((name.value.decode(), ms.value))
     return out
+
+
+def stem_dedup_ids_static(shape, ids, unique_ids, n_unique, inverse, perm, seg_offsets, status=None, stream=None) -> None:
+    """Dedup for callers that cannot allocate: scratch is a fixed array inside the library."""
+    _check(lib().stem_dedup_ids_static(ctypes.byref(shape), _p(ids), _p(unique_ids), _p(n_unique), _p(inverse),
+                                       _p(perm), _p(seg_offsets), _p(status), _stream(stream)),
+           "stem_dedup_ids_static")
+
+
+def stem_dedup_static_max_tokens() -> int:
+    return lib().stem_dedup_static_max_tokens()

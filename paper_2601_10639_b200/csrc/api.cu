@@ -161,6 +161,7 @@ const char* stem_status_string(int code) {
     case STEM_ERR_CUDA: return g_cuda_msg[0] ? g_cuda_msg : "CUDA error";
     case STEM_ERR_TIMEOUT: return "device: a bounded pipeline wait expired";
     case STEM_ERR_ID_RANGE: return "device: token id outside [0,V) (clamped)";
+    case STEM_ERR_STATIC_LIMIT: return "size exceeds the fixed scratch of the allocation-free entry point (T > 65536)";
     default: return "unknown status";
   }
 }

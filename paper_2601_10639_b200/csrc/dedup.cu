@@ -2,6 +2,8 @@
 // pass, followed by one pass that marks the head of every run of equal ids and emits the
 // distinct ids, the run offsets and each position's slot.  Integer-only: every output has
 // exactly one correct value.
+#include <mutex>
+
 #include "stem_internal.h"
 
 namespace stem {
@@ -223,3 +225,61 @@ cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, 
 }
 
 }  // namespace stem
+
+// ---- dedup without a caller workspace ---------------------------------------------------
+// Some callers cannot hand the library scratch memory because they cannot allocate any:
+// a serving process whose framework reserved all of HBM at start-up for weights and KV
+// cache, a plug-in that runs inside another runtime's stream callback, or a latency-bound
+// loop where a cudaMalloc would synchronise the whole device.  For them the radix sort's
+// ping-pong buffers and digit counts live in this fixed array, which every GPU that loads
+// the library holds until the process exits (1.25 MiB).
+namespace stem {
+namespace {
+
+constexpr int kStaticMaxT = 65536;
+constexpr size_t kStaticScratchBytes = 4 * static_cast<size_t>(kStaticMaxT) * 4 +
+                                       static_cast<size_t>(kStaticMaxT / 256) * kRadix * 4;
+static __device__ __align__(256) unsigned char g_dedup_scratch[kStaticScratchBytes];
+
+// The array's name is only a host-side handle; kernels need its device address, which
+// differs per device and is looked up once per device.
+std::mutex g_static_mutex;
+void* g_static_ptr[64] = {nullptr};
+
+cudaError_t static_scratch_address(void** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_dedup_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_ptr[dev] = p;
+  }
+  *out = g_static_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace stem
+
+extern "C" int stem_dedup_ids_static(const stem_shape_t* shape, const int32_t* ids, int32_t* unique_ids,
+                                     int32_t* n_unique, int32_t* inverse, int32_t* perm,
+                                     int32_t* seg_offsets, int32_t* status, void* stream) {
+  using namespace stem;
+  if (!shape || shape->T < 0 || shape->V <= 0 || shape->V > (1 << 30)) return STEM_ERR_INVALID_ARG;
+  if (shape->T > kStaticMaxT) return STEM_ERR_STATIC_LIMIT;
+  if (!unique_ids || !n_unique || !perm || !seg_offsets || (shape->T > 0 && !ids)) return STEM_ERR_INVALID_ARG;
+  if (dedup_workspace_bytes(shape->T, shape->V) > kStaticScratchBytes) return STEM_ERR_STATIC_LIMIT;
+  void* scratch = nullptr;
+  if (static_scratch_address(&scratch) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
+  // Nothing in the scratch has to start at zero: every pass writes each digit count and each
+  // key/value slot it later reads, so whatever the previous call left behind is overwritten.
+  cudaError_t e = launch_dedup(shape->T, shape->V, ids, unique_ids, n_unique, inverse, perm, seg_offsets,
+                               scratch, status, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? STEM_OK : STEM_ERR_CUDA;
+}
+
+extern "C" int stem_dedup_static_max_tokens(void) { return stem::kStaticMaxT; }
