@@ -8,8 +8,11 @@
 //   warp 0      one thread issues TMA loads into a STAGES-deep shared-memory ring
 //   warp 1      allocates TMEM; one thread issues tcgen05.mma (128 x BN x 16 per
 //               instruction, four per 64-wide k block) and commits to mbarriers
-//   warps 2..5  epilogue: tcgen05.ld the finished 128 x BN fp32 tile (one row per thread),
-//               apply the fused elementwise step, store
+//   warps 2..9  epilogue: tcgen05.ld the finished 128 x BN fp32 tile (one row per thread,
+//               two warps per TMEM lane quarter, each taking half of the columns), apply
+//               the fused elementwise step, store.  The table row and the saved G are
+//               fetched one 32-column chunk ahead of the arithmetic, with 32-byte
+//               accesses, so their latency hides behind the previous chunk
 // Two accumulator tiles live in TMEM (2 x BN columns), so the epilogue of tile i overlaps
 // the MMAs of tile i+1.  Operands may be K-major or MN-major (the backward pass contracts
 // over the token dimension, which is the slow index of every [T, .] tensor); both use the
@@ -29,7 +32,7 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int UMMA_K = 16;
-constexpr int kEpiWarps = 4;
+constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr long long kWaitLimitCycles = 2000000000ll;  // ~1 s at boost clock
 constexpr int kAtomBytes = 64 * BK * 2;                // one 64(MN) x BK swizzled block
@@ -49,66 +52,103 @@ __device__ __forceinline__ float fast_sigmoid(float g) {
   return __fdividef(1.0f, 1.0f + __expf(-g));
 }
 
-__device__ __forceinline__ void unpack_bf16x8(const uint4& q, float (&v)[8]) {
-  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-  }
+// ---- 32-column row segments: global <-> registers -------------------------------------
+// WIDE: the row pitch and base are multiples of 32 bytes, so 256-bit accesses are legal and
+// a 16-column group is wholly inside or outside the matrix.  Otherwise 128-bit accesses.
+__device__ __forceinline__ void ldg256(const void* p, uint32_t* r) {
+  asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "l"(p));
 }
-__device__ __forceinline__ uint4 pack_bf16x8(const float (&v)[8]) {
-  uint32_t w[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-    w[i] = *reinterpret_cast<const uint32_t*>(&h);
-  }
-  return make_uint4(w[0], w[1], w[2], w[3]);
+__device__ __forceinline__ void stg256(void* p, const uint32_t* r) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+__device__ __forceinline__ void ldg128(const void* p, uint32_t* r) {
+  const uint4 q = __ldg(static_cast<const uint4*>(p));
+  r[0] = q.x; r[1] = q.y; r[2] = q.z; r[3] = q.w;
+}
+__device__ __forceinline__ void stg128(void* p, const uint32_t* r) {
+  *static_cast<uint4*>(p) = make_uint4(r[0], r[1], r[2], r[3]);
 }
 
-// Fused elementwise step on 32 consecutive columns of one output row.
-template <int KIND>
-__device__ __forceinline__ void epilogue_row32(const EpiParams& ep, bool row_ok, size_t row_off,
-                                               const __nv_bfloat16* e_row, int n, int N,
-                                               const uint32_t (&acc)[32]) {
-  if (!row_ok) return;
+// 32 bf16 (16 registers) starting at column n of a row; p points at column n.
+template <bool WIDE>
+__device__ __forceinline__ void load_bf16x32(const __nv_bfloat16* p, int n, int N, uint32_t (&r)[16]) {
+  if (WIDE) {
 #pragma unroll
-  for (int g8 = 0; g8 < 4; ++g8) {
-    const int nn = n + g8 * 8;
-    if (nn >= N) break;  // N is a multiple of 8: a group is wholly in or wholly out
-    float a[8];
+    for (int h = 0; h < 2; ++h) if (n + 16 * h < N) ldg256(p + 16 * h, r + 8 * h);
+  } else {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) a[i] = __uint_as_float(acc[g8 * 8 + i]);
-    if (KIND == kEpiStore) {
-      if (ep.out_fp32) {
-        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(ep.out) + row_off + nn);
-        dst[0] = make_float4(a[0], a[1], a[2], a[3]);
-        dst[1] = make_float4(a[4], a[5], a[6], a[7]);
-      } else {
-        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.out) + row_off + nn) = pack_bf16x8(a);
-      }
-    } else if (KIND == kEpiGate) {
-      float u[8], h[8];
-      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(e_row + nn)), u);
+    for (int q = 0; q < 4; ++q) if (n + 8 * q < N) ldg128(p + 8 * q, r + 4 * q);
+  }
+}
+template <bool WIDE>
+__device__ __forceinline__ void store_bf16x32(__nv_bfloat16* p, int n, int N, const uint32_t (&r)[16]) {
+  if (WIDE) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) h[i] = a[i] * fast_sigmoid(a[i]) * u[i];
-      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.H) + row_off + nn) = pack_bf16x8(h);
-      if (ep.G)
-        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.G) + row_off + nn) = pack_bf16x8(a);
+    for (int h = 0; h < 2; ++h) if (n + 16 * h < N) stg256(p + 16 * h, r + 8 * h);
+  } else {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) if (n + 8 * q < N) stg128(p + 8 * q, r + 4 * q);
+  }
+}
+template <bool WIDE>
+__device__ __forceinline__ void store_f32x32(float* p, int n, int N, const uint32_t (&r)[32]) {
+  if (WIDE) {
+#pragma unroll
+    for (int h = 0; h < 4; ++h) if (n + 8 * h < N) stg256(p + 8 * h, r + 8 * h);
+  } else {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) if (n + 4 * q < N) stg128(p + 4 * q, r + 4 * q);
+  }
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// Fused elementwise step on 32 consecutive columns of one output row.  e and g hold the
+// table row segment and the saved pre-activation (bf16 pairs), fetched earlier.
+template <int KIND, bool WIDE>
+__device__ __forceinline__ void epilogue_row32(const EpiParams& ep, size_t off, int n, int N,
+                                               const uint32_t (&acc)[32], const uint32_t (&e)[16],
+                                               const uint32_t (&g)[16]) {
+  if (KIND == kEpiStore) {
+    if (ep.out_fp32) {
+      store_f32x32<WIDE>(static_cast<float*>(ep.out) + off, n, N, acc);
     } else {
-      float u[8], g[8], du[8], dg[8];
-      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(e_row + nn)), u);
-      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(ep.Gin) + row_off + nn)), g);
+      uint32_t o[16];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float s = fast_sigmoid(g[i]);
-        du[i] = a[i] * (g[i] * s);
-        dg[i] = a[i] * u[i] * (s * (1.0f + g[i] * (1.0f - s)));
-      }
-      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.H) + row_off + nn) = pack_bf16x8(du);
-      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.G) + row_off + nn) = pack_bf16x8(dg);
+      for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
+      store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.out) + off, n, N, o);
     }
+  } else if (KIND == kEpiGate) {
+    uint32_t h[16], go[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float a0 = __uint_as_float(acc[2 * i]), a1 = __uint_as_float(acc[2 * i + 1]);
+      h[i] = pack_bf16(a0 * fast_sigmoid(a0) * bf16_lo(e[i]), a1 * fast_sigmoid(a1) * bf16_hi(e[i]));
+      go[i] = pack_bf16(a0, a1);
+    }
+    store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.H) + off, n, N, h);
+    if (ep.G) store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.G) + off, n, N, go);
+  } else {
+    uint32_t du[16], dg[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float a0 = __uint_as_float(acc[2 * i]), a1 = __uint_as_float(acc[2 * i + 1]);
+      const float g0 = bf16_lo(g[i]), g1 = bf16_hi(g[i]);
+      const float s0 = fast_sigmoid(g0), s1 = fast_sigmoid(g1);
+      du[i] = pack_bf16(a0 * (g0 * s0), a1 * (g1 * s1));
+      dg[i] = pack_bf16(a0 * bf16_lo(e[i]) * (s0 * (1.0f + g0 * (1.0f - s0))),
+                        a1 * bf16_hi(e[i]) * (s1 * (1.0f + g1 * (1.0f - s1))));
+    }
+    store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.H) + off, n, N, du);
+    store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.G) + off, n, N, dg);
   }
 }
 
@@ -122,7 +162,7 @@ __device__ __forceinline__ TileCoord tile_coord(int tile, int tiles_m, int tiles
   return {first_m + in % gsize, in / gsize};
 }
 
-template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES>
+template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                int M, int N, int K, int group_m, EpiParams ep) {
@@ -246,16 +286,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else {
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;       // which half of the tile's columns it handles
+    constexpr int kChunks = BN / 2 / 32;    // 32-column chunks per thread per tile
     int acc = 0; uint32_t aph = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       const TileCoord tc = tile_coord(tile, tiles_m, tiles_n, group_m);
       const int m = tc.m_blk * BM + q * 32 + lane;
-      const int n0 = tc.n_blk * BN;
+      const int n0 = tc.n_blk * BN + half * (BN / 2);
       const bool row_ok = m < M;
       const size_t row_off = static_cast<size_t>(m) * N;
       const __nv_bfloat16* e_row = nullptr;
+      const __nv_bfloat16* g_row = nullptr;
       if (KIND != kEpiStore && row_ok) {
         int id = ep.ids[m];
         if (id < 0 || id >= ep.V) {
@@ -263,6 +306,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           id = id < 0 ? 0 : ep.V - 1;
         }
         e_row = static_cast<const __nv_bfloat16*>(ep.E) + static_cast<size_t>(id) * N;
+        if (KIND == kEpiDH) g_row = static_cast<const __nv_bfloat16*>(ep.Gin) + row_off;
+      }
+      // operands of the first chunk are requested before waiting for the accumulator
+      uint32_t e_next[16], g_next[16];
+      if (KIND != kEpiStore && row_ok) {
+        load_bf16x32<WIDE>(e_row + n0, n0, N, e_next);
+        if (KIND == kEpiDH) load_bf16x32<WIDE>(g_row + n0, n0, N, g_next);
       }
       bool mine = ptx::mbar_wait_bounded(tfull_bar(acc), aph, abort_flag, kWaitLimitCycles);
       mine = __all_sync(0xffffffffu, mine);
@@ -271,13 +321,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         ok = false; break;
       }
       ptx::tc_fence_after();
-      const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(q * 32) << 16);
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      const uint32_t t_row = tmem_base + acc * BN + half * (BN / 2) + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll
+      for (int c = 0; c < kChunks; ++c) {
+        uint32_t e_cur[16], g_cur[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) { e_cur[i] = e_next[i]; g_cur[i] = g_next[i]; }
+        const int n = n0 + c * 32;
+        if (KIND != kEpiStore && row_ok && c + 1 < kChunks) {
+          load_bf16x32<WIDE>(e_row + n + 32, n + 32, N, e_next);
+          if (KIND == kEpiDH) load_bf16x32<WIDE>(g_row + n + 32, n + 32, N, g_next);
+        }
         uint32_t v[32];
         ptx::tmem_ld_32x32(t_row + c * 32, v);
         ptx::tmem_ld_wait();
-        epilogue_row32<KIND>(ep, row_ok, row_off, e_row, n0 + c * 32, N, v);
+        if (row_ok) epilogue_row32<KIND, WIDE>(ep, row_off + n, n, N, v, e_cur, g_cur);
       }
       ptx::tc_fence_before();
       __syncwarp();
@@ -335,11 +393,11 @@ bool encode_map(CUtensorMap* map, const void* ptr, int rows, int cols, int box_r
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES>
+template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE>
 cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, int M, int N, int K,
                         const EpiParams& ep, cudaStream_t stream) {
   using L = Smem<BN, STAGES>;
-  auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES>;
+  auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES, WIDE>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
@@ -361,7 +419,10 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
   const bool okA = A_MN ? encode_map(&tmA, A, K, M, BK) : encode_map(&tmA, A, M, K, BM);
   const bool okB = B_MN ? encode_map(&tmB, B, K, N, BK) : encode_map(&tmB, B, N, K, BN);
   if (!okA || !okB) return cudaErrorNotSupported;
-  return launch_inst<A_MN, B_MN, KIND, BN, STAGES>(tmA, tmB, M, N, K, ep, stream);
+  auto a32 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; };
+  const bool wide = (N % 16 == 0) && a32(ep.out) && a32(ep.E) && a32(ep.H) && a32(ep.G) && a32(ep.Gin);
+  if (wide) return launch_inst<A_MN, B_MN, KIND, BN, STAGES, true>(tmA, tmB, M, N, K, ep, stream);
+  return launch_inst<A_MN, B_MN, KIND, BN, STAGES, false>(tmA, tmB, M, N, K, ep, stream);
 }
 
 }  // namespace
