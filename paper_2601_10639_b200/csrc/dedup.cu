@@ -1,7 +1,7 @@
 // Token-id deduplication: a stable LSD radix sort of (id, position) pairs, 8 bits per
-// pass, followed by one pass that marks the head of every run of equal ids and emits the
-// distinct ids, the run offsets and each position's slot.  Integer-only: every output has
-// exactly one correct value.
+// pass (a count kernel and a scatter kernel per pass), followed by two kernels that mark
+// the head of every run of equal ids and emit the distinct ids, the run offsets and each
+// position's slot.  Integer-only: every output has exactly one correct value.
 #include <mutex>
 
 #include "stem_internal.h"
@@ -10,83 +10,99 @@ namespace stem {
 namespace {
 
 constexpr int kRadix = 256;
-constexpr int kWarpsPerBlock = 8;
+constexpr int kWarps = 32;              // warps per CTA
+constexpr int kCtaThreads = kWarps * 32;
+constexpr int kMaxCtas = 64;
 
-__host__ __device__ inline int elems_per_warp(int T) { return T <= (1 << 16) ? 256 : 2048; }
+// Work split: CTA c owns positions [c * 32 * epw, (c + 1) * 32 * epw), warp w of it the
+// w-th run of epw positions.  Few, large CTAs keep the cross-CTA bookkeeping (one digit
+// histogram per CTA) small enough for every CTA to re-derive its offsets by itself.
+struct Split { int n_ctas, epw; };
+__host__ __device__ inline Split make_split(int T) {
+  int n_ctas = (T + 4095) / 4096;
+  n_ctas = n_ctas < 1 ? 1 : (n_ctas > kMaxCtas ? kMaxCtas : n_ctas);
+  const int per_cta = (T + n_ctas - 1) / n_ctas;
+  const int epw = ((per_cta + kWarps - 1) / kWarps + 31) / 32 * 32;
+  return {n_ctas, epw};
+}
 
-// Each warp owns a contiguous run of positions; counts[digit * n_warps + warp] = how many
-// of its keys carry `digit` at `shift`.
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
-radix_count_kernel(int T, int V, int epw, int n_warps, int shift, bool first_pass,
-                   const int32_t* __restrict__ keys_in, int32_t* __restrict__ counts,
-                   int32_t* status) {
-  __shared__ int hist[kWarpsPerBlock][kRadix];
+__device__ __forceinline__ int clamp_id(int key, int V) { return key < 0 ? 0 : (key >= V ? V - 1 : key); }
+
+// Per-warp digit histograms of this CTA's keys, in shared memory.
+__device__ __forceinline__ void warp_histograms(int (*hist)[kRadix], int T, int V, int epw, int shift,
+                                                bool first_pass, const int32_t* __restrict__ keys_in,
+                                                int32_t* status) {
   const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int i = lane; i < kRadix; i += 32) hist[w][i] = 0;
   __syncwarp();
-  const int gw = blockIdx.x * kWarpsPerBlock + w;
-  if (gw < n_warps) {
-    const int begin = gw * epw, end = min(T, begin + epw);
-    for (int i = begin + lane; i < end; i += 32) {
-      int key = keys_in[i];
-      if (first_pass && (key < 0 || key >= V)) {
-        if (status) { report_error(status, STEM_ERR_ID_RANGE, i); atomicAdd(status + 2, 1); }
-        key = key < 0 ? 0 : V - 1;
+  const int begin = (blockIdx.x * kWarps + w) * epw, end = min(T, begin + epw);
+  for (int i = begin + lane; i < end; i += 32) {
+    int key = keys_in[i];
+    if (first_pass) {
+      if (status != nullptr && (key < 0 || key >= V)) {
+        report_error(status, STEM_ERR_ID_RANGE, i);
+        atomicAdd(status + 2, 1);
       }
-      atomicAdd(&hist[w][(key >> shift) & (kRadix - 1)], 1);
+      key = clamp_id(key, V);
     }
-    __syncwarp();
-    for (int d = lane; d < kRadix; d += 32) counts[d * n_warps + gw] = hist[w][d];
+    atomicAdd(&hist[w][(key >> shift) & (kRadix - 1)], 1);
   }
 }
 
-// Exclusive prefix sum of n ints in place, one block.
-__global__ void __launch_bounds__(1024) scan_exclusive_kernel(int32_t* data, int n) {
-  __shared__ int warp_sums[32];
-  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-  const int per = (n + 1023) / 1024;
-  const int begin = min(n, tid * per), end = min(n, begin + per);
-  int local = 0;
-  for (int i = begin; i < end; ++i) local += data[i];
-  int incl = local;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int v = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += v;
-  }
-  if (lane == 31) warp_sums[w] = incl;
+// cta_hist[c][d] = number of keys of CTA c whose digit at `shift` is d.
+__global__ void __launch_bounds__(kCtaThreads)
+radix_count_kernel(int T, int V, int epw, int shift, bool first_pass, const int32_t* __restrict__ keys_in,
+                   int32_t* __restrict__ cta_hist, int32_t* status) {
+  __shared__ int hist[kWarps][kRadix];
+  warp_histograms(hist, T, V, epw, shift, first_pass, keys_in, status);
   __syncthreads();
-  if (w == 0) {
-    int s = warp_sums[lane];
+  if (threadIdx.x < kRadix) {
+    int sum = 0;
+#pragma unroll 8
+    for (int w = 0; w < kWarps; ++w) sum += hist[w][threadIdx.x];
+    cta_hist[blockIdx.x * kRadix + threadIdx.x] = sum;
+  }
+}
+
+// Stable scatter.  Every CTA derives its own output offsets from all CTAs' histograms:
+// keys with a smaller digit first, then equal digits of earlier CTAs, then of earlier warps.
+__global__ void __launch_bounds__(kCtaThreads)
+radix_scatter_kernel(int T, int V, int epw, int shift, bool first_pass, const int32_t* __restrict__ keys_in,
+                     const int32_t* __restrict__ vals_in, const int32_t* __restrict__ cta_hist,
+                     int32_t* __restrict__ keys_out, int32_t* __restrict__ vals_out) {
+  __shared__ int hist[kWarps][kRadix];
+  __shared__ int warp_tot[kRadix / 32];
+  warp_histograms(hist, T, V, epw, shift, first_pass, keys_in, nullptr);
+  __syncthreads();
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int before = 0, total = 0;
+  if (threadIdx.x < kRadix) {
+    for (int c = 0; c < static_cast<int>(gridDim.x); ++c) {
+      const int v = cta_hist[c * kRadix + threadIdx.x];
+      total += v;
+      if (c < static_cast<int>(blockIdx.x)) before += v;
+    }
+    int incl = total;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int v = __shfl_up_sync(0xffffffffu, s, o);
-      if (lane >= o) s += v;
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
     }
-    warp_sums[lane] = s;
+    if (lane == 31) warp_tot[w] = incl;
+    total = incl - total;  // exclusive prefix inside this warp of digits
   }
   __syncthreads();
-  int run = incl - local + (w > 0 ? warp_sums[w - 1] : 0);
-  for (int i = begin; i < end; ++i) {
-    const int v = data[i];
-    data[i] = run;
-    run += v;
+  if (threadIdx.x < kRadix) {
+    int base = total + before;
+    for (int ww = 0; ww < w; ++ww) base += warp_tot[ww];
+    for (int ww = 0; ww < kWarps; ++ww) {  // turn per-warp counts into per-warp start offsets
+      const int cnt = hist[ww][threadIdx.x];
+      hist[ww][threadIdx.x] = base;
+      base += cnt;
+    }
   }
-}
-
-// Stable scatter: within a warp's run, keys with the same digit keep their order.
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
-radix_scatter_kernel(int T, int V, int epw, int n_warps, int shift, bool first_pass,
-                     const int32_t* __restrict__ keys_in, const int32_t* __restrict__ vals_in,
-                     const int32_t* __restrict__ offsets, int32_t* __restrict__ keys_out,
-                     int32_t* __restrict__ vals_out) {
-  __shared__ int base[kWarpsPerBlock][kRadix];
-  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int gw = blockIdx.x * kWarpsPerBlock + w;
-  if (gw >= n_warps) return;
-  for (int d = lane; d < kRadix; d += 32) base[w][d] = offsets[d * n_warps + gw];
-  __syncwarp();
-  const int begin = gw * epw, end = min(T, begin + epw);
+  __syncthreads();
+  const int begin = (blockIdx.x * kWarps + w) * epw, end = min(T, begin + epw);
   const unsigned lt_mask = (1u << lane) - 1u;
   for (int i0 = begin; i0 < end; i0 += 32) {
     const int i = i0 + lane;
@@ -94,41 +110,61 @@ radix_scatter_kernel(int T, int V, int epw, int n_warps, int shift, bool first_p
     int key = 0, val = 0;
     if (valid) {
       key = keys_in[i];
-      if (first_pass) {
-        key = key < 0 ? 0 : (key >= V ? V - 1 : key);
-        val = i;
-      } else {
-        val = vals_in[i];
-      }
+      if (first_pass) { key = clamp_id(key, V); val = i; } else { val = vals_in[i]; }
     }
     const int digit = (key >> shift) & (kRadix - 1);
     const unsigned peers = __match_any_sync(0xffffffffu, valid ? digit : (kRadix + lane));
     const int rank = __popc(peers & lt_mask);
     int dst = 0;
-    if (valid) dst = base[w][digit] + rank;
+    if (valid) dst = hist[w][digit] + rank;
     __syncwarp();
-    if (valid && rank == 0) base[w][digit] += __popc(peers);
+    if (valid && rank == 0) hist[w][digit] += __popc(peers);
     __syncwarp();
-    if (valid) {
-      keys_out[dst] = key;
-      vals_out[dst] = val;
-    }
+    if (valid) { keys_out[dst] = key; vals_out[dst] = val; }
   }
 }
 
-// One block walks the sorted ids: heads of runs -> unique_ids / seg_offsets, slot of every
-// position -> inverse.
-__global__ void __launch_bounds__(1024)
-segment_heads_kernel(int T, const int32_t* __restrict__ sorted_ids, const int32_t* __restrict__ perm,
-                     int32_t* __restrict__ unique_ids, int32_t* __restrict__ n_unique,
-                     int32_t* __restrict__ inverse, int32_t* __restrict__ seg_offsets) {
-  __shared__ int warp_sums[32];
-  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-  const int per = (T + 1023) / 1024;
-  const int begin = min(T, tid * per), end = min(T, begin + per);
+__device__ __forceinline__ bool is_head(const int32_t* __restrict__ sorted_ids, int p) {
+  return p == 0 || sorted_ids[p] != sorted_ids[p - 1];
+}
+
+// Heads of runs of equal ids, counted per CTA chunk.
+__global__ void __launch_bounds__(kCtaThreads)
+heads_count_kernel(int T, int per_cta, const int32_t* __restrict__ sorted_ids, int32_t* __restrict__ cta_heads) {
+  const int begin = blockIdx.x * per_cta, end = min(T, begin + per_cta);
   int local = 0;
-  for (int p = begin; p < end; ++p)
-    local += (p == 0 || sorted_ids[p] != sorted_ids[p - 1]) ? 1 : 0;
+  for (int p = begin + threadIdx.x; p < end; p += kCtaThreads) local += is_head(sorted_ids, p) ? 1 : 0;
+  __shared__ int s_sum;
+  if (threadIdx.x == 0) s_sum = 0;
+  __syncthreads();
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xffffffffu, local, o);
+  if ((threadIdx.x & 31) == 0 && local) atomicAdd(&s_sum, local);
+  __syncthreads();
+  if (threadIdx.x == 0) cta_heads[blockIdx.x] = s_sum;
+}
+
+// unique_ids / seg_offsets at the heads, slot of every position -> inverse.
+__global__ void __launch_bounds__(kCtaThreads)
+heads_write_kernel(int T, int per_cta, const int32_t* __restrict__ sorted_ids, const int32_t* __restrict__ perm,
+                   const int32_t* __restrict__ cta_heads, int32_t* __restrict__ unique_ids,
+                   int32_t* __restrict__ n_unique, int32_t* __restrict__ inverse,
+                   int32_t* __restrict__ seg_offsets) {
+  __shared__ int warp_sums[kWarps];
+  __shared__ int s_before;
+  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+  if (w == 0) {
+    int v = 0;
+    for (int c = lane; c < static_cast<int>(blockIdx.x); c += 32) v += cta_heads[c];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == 0) s_before = v;
+  }
+  const int cta_begin = blockIdx.x * per_cta, cta_end = min(T, cta_begin + per_cta);
+  const int per_thread = (per_cta + kCtaThreads - 1) / kCtaThreads;
+  const int begin = min(cta_end, cta_begin + tid * per_thread), end = min(cta_end, begin + per_thread);
+  int local = 0;
+  for (int p = begin; p < end; ++p) local += is_head(sorted_ids, p) ? 1 : 0;
   int incl = local;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -138,27 +174,27 @@ segment_heads_kernel(int T, const int32_t* __restrict__ sorted_ids, const int32_
   if (lane == 31) warp_sums[w] = incl;
   __syncthreads();
   if (w == 0) {
-    int s = warp_sums[lane];
+    int v = warp_sums[lane];
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int v = __shfl_up_sync(0xffffffffu, s, o);
-      if (lane >= o) s += v;
+      const int u = __shfl_up_sync(0xffffffffu, v, o);
+      if (lane >= o) v += u;
     }
-    warp_sums[lane] = s;
+    warp_sums[lane] = v;
   }
   __syncthreads();
-  int heads_before = incl - local + (w > 0 ? warp_sums[w - 1] : 0);
+  int heads = s_before + incl - local + (w > 0 ? warp_sums[w - 1] : 0);  // heads before `begin`
   for (int p = begin; p < end; ++p) {
     const int id = sorted_ids[p];
-    if (p == 0 || id != sorted_ids[p - 1]) {
-      unique_ids[heads_before] = id;
-      seg_offsets[heads_before] = p;
-      ++heads_before;
+    if (is_head(sorted_ids, p)) {
+      unique_ids[heads] = id;
+      seg_offsets[heads] = p;
+      ++heads;
     }
-    if (inverse) inverse[perm[p]] = heads_before - 1;
+    if (inverse) inverse[perm[p]] = heads - 1;
   }
-  if (tid == 1023) {
-    const int total = warp_sums[31];
+  if (blockIdx.x == gridDim.x - 1 && tid == 0) {
+    const int total = s_before + warp_sums[kWarps - 1];
     *n_unique = total;
     seg_offsets[total] = T;
   }
@@ -180,10 +216,8 @@ int key_bits(int V) {
 size_t dedup_workspace_bytes(int T, int V) {
   (void)V;
   if (T <= 0) return 0;
-  const int epw = elems_per_warp(T);
-  const int n_warps = (T + epw - 1) / epw;
-  // two key buffers, two value buffers, the digit counts
-  return 4 * align_up(static_cast<size_t>(T) * 4, 256) + align_up(static_cast<size_t>(n_warps) * kRadix * 4, 256);
+  // two key buffers, two value buffers, per-CTA digit histograms, per-CTA head counts
+  return 4 * align_up(static_cast<size_t>(T) * 4, 256) + static_cast<size_t>(kMaxCtas) * kRadix * 4 + 256;
 }
 
 cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, int32_t* n_unique,
@@ -194,33 +228,33 @@ cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, 
     count_launches(1);
     return cudaGetLastError();
   }
-  const int epw = elems_per_warp(T);
-  const int n_warps = (T + epw - 1) / epw;
+  const Split sp = make_split(T);
   const size_t tb = align_up(static_cast<size_t>(T) * 4, 256);
   char* p = static_cast<char*>(scratch);
   int32_t* keys[2] = {reinterpret_cast<int32_t*>(p), reinterpret_cast<int32_t*>(p + tb)};
   int32_t* vals[2] = {reinterpret_cast<int32_t*>(p + 2 * tb), reinterpret_cast<int32_t*>(p + 3 * tb)};
-  int32_t* counts = reinterpret_cast<int32_t*>(p + 4 * tb);
+  int32_t* cta_hist = reinterpret_cast<int32_t*>(p + 4 * tb);
+  int32_t* cta_heads = cta_hist + kMaxCtas * kRadix;
 
   const int passes = (key_bits(V) + 7) / 8;
-  const int blocks = (n_warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
   const int32_t* kin = ids;
   const int32_t* vin = nullptr;
   for (int pass = 0; pass < passes; ++pass) {
     const bool first = pass == 0, last = pass == passes - 1;
     int32_t* kout = keys[pass & 1];
     int32_t* vout = last ? perm : vals[pass & 1];
-    radix_count_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(T, V, epw, n_warps, pass * 8, first,
-                                                                  kin, counts, status);
-    scan_exclusive_kernel<<<1, 1024, 0, stream>>>(counts, n_warps * kRadix);
-    radix_scatter_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(T, V, epw, n_warps, pass * 8, first,
-                                                                    kin, vin, counts, kout, vout);
-    count_launches(3);
+    radix_count_kernel<<<sp.n_ctas, kCtaThreads, 0, stream>>>(T, V, sp.epw, pass * 8, first, kin, cta_hist, status);
+    radix_scatter_kernel<<<sp.n_ctas, kCtaThreads, 0, stream>>>(T, V, sp.epw, pass * 8, first, kin, vin, cta_hist,
+                                                               kout, vout);
+    count_launches(2);
     kin = kout;
     vin = vout;
   }
-  segment_heads_kernel<<<1, 1024, 0, stream>>>(T, kin, perm, unique_ids, n_unique, inverse, seg_offsets);
-  count_launches(1);
+  const int per_cta = sp.epw * kWarps;
+  heads_count_kernel<<<sp.n_ctas, kCtaThreads, 0, stream>>>(T, per_cta, kin, cta_heads);
+  heads_write_kernel<<<sp.n_ctas, kCtaThreads, 0, stream>>>(T, per_cta, kin, perm, cta_heads, unique_ids, n_unique,
+                                                           inverse, seg_offsets);
+  count_launches(2);
   return cudaGetLastError();
 }
 
@@ -237,8 +271,7 @@ namespace stem {
 namespace {
 
 constexpr int kStaticMaxT = 65536;
-constexpr size_t kStaticScratchBytes = 4 * static_cast<size_t>(kStaticMaxT) * 4 +
-                                       static_cast<size_t>(kStaticMaxT / 256) * kRadix * 4;
+constexpr size_t kStaticScratchBytes = 1310720;  // 1.25 MiB >= dedup_workspace_bytes(kStaticMaxT, .)
 static __device__ __align__(256) unsigned char g_dedup_scratch[kStaticScratchBytes];
 
 // The array's name is only a host-side handle; kernels need its device address, which

@@ -5,42 +5,47 @@
 // per (block, column slab) walks its positions in order, accumulating in fp32 registers.
 // A run whose segment lies wholly inside the block is final and is written to dE_rows; a
 // run whose segment crosses a block edge (at most the first and the last run of a block)
-// goes to a partial row.  Pass 2: the CTA of the block in which a crossing segment starts
-// adds that segment's partial rows in block order.  Both orders depend on the index arrays
-// only, so the result is bitwise reproducible.  HBM-bound: every dU row is read once with
-// 16-byte loads, coalesced along d_ff.
+// goes to a partial row, and the block in which such a segment starts is appended to a
+// list.  Pass 2: one CTA per list entry adds that segment's partial rows.  The order of the
+// list varies from run to run (an integer atomic hands out its slots) but each entry is
+// handled on its own and every summation order depends on the index arrays only, so the
+// result is bitwise reproducible.  HBM-bound: every dU row is read once with 16-byte loads,
+// coalesced along d_ff.
 #include "stem_internal.h"
 
 namespace stem {
 namespace {
 
-constexpr int kSegBlk = 64;
-constexpr int kThreads = 256;
-constexpr int kBatch = 8;
+constexpr int kSegBlk = 64;     // sorted positions per CTA of pass 1
+constexpr int kThreads = 128;   // pass 1: one thread per vector of columns
+constexpr int kBatch = 8;       // rows requested before the first is consumed
+constexpr int kRowLanes = 8;    // pass 2: partial rows summed side by side
+constexpr int kColLanes = 32;
 
 template <typename T> struct Vec;
 template <> struct Vec<float> {
   static constexpr int N = 4;
-  __device__ static void load(const float* p, float (&v)[4]) {
-    const float4 q = __ldg(reinterpret_cast<const float4*>(p));
-    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+  __device__ static uint4 load_raw(const float* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ static void add(float* acc, const uint4& q) {
+    acc[0] += __uint_as_float(q.x); acc[1] += __uint_as_float(q.y);
+    acc[2] += __uint_as_float(q.z); acc[3] += __uint_as_float(q.w);
   }
-  __device__ static void store(float* p, const float (&v)[4]) {
+  __device__ static void store(float* p, const float* v) {
     *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
   }
 };
 template <> struct Vec<__nv_bfloat16> {
   static constexpr int N = 8;
-  __device__ static void load(const __nv_bfloat16* p, float (&v)[8]) {
-    const uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
+  __device__ static uint4 load_raw(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ static void add(float* acc, const uint4& q) {
     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      v[2 * i] = __uint_as_float(w[i] << 16);
-      v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+      acc[2 * i] += __uint_as_float(w[i] << 16);
+      acc[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
     }
   }
-  __device__ static void store(__nv_bfloat16* p, const float (&v)[8]) {
+  __device__ static void store(__nv_bfloat16* p, const float* v) {
     uint32_t w[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -51,51 +56,70 @@ template <> struct Vec<__nv_bfloat16> {
   }
 };
 
-// largest r in [0, n_u) with seg_offsets[r] <= p   (p < T = seg_offsets[n_u])
-__device__ __forceinline__ int segment_of(const int32_t* seg_offsets, int n_u, int p) {
-  int lo = 0, hi = n_u;  // invariant: seg_offsets[lo] <= p < seg_offsets[hi]
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (seg_offsets[mid] <= p) lo = mid; else hi = mid;
-  }
-  return lo;
-}
-
 // A thread owns VI consecutive columns; rows are written in the output type's vectors.
 template <int VI, typename TOut>
 __device__ __forceinline__ void store_row(TOut* dst, const float (&v)[VI]) {
 #pragma unroll
-  for (int i = 0; i < VI; i += Vec<TOut>::N) {
-    float t[Vec<TOut>::N];
-#pragma unroll
-    for (int j = 0; j < Vec<TOut>::N; ++j) t[j] = v[i + j];
-    Vec<TOut>::store(dst + i, t);
-  }
+  for (int i = 0; i < VI; i += Vec<TOut>::N) Vec<TOut>::store(dst + i, v + i);
+}
+
+// Scratch layout: [0] number of entries in the list of crossing segments, [1..n_blk] the
+// list (block in which each crossing segment starts), then 2 partial rows per block.
+__host__ __device__ inline size_t partial_offset_bytes(int n_blk) {
+  return (static_cast<size_t>(n_blk + 1) * 4 + 255) / 256 * 256;
 }
 
 template <typename TIn, typename TOut>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 6)
 segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* __restrict__ perm,
                        const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ n_unique,
-                       TOut* __restrict__ dE_rows, float* __restrict__ partial) {
+                       TOut* __restrict__ dE_rows, int32_t* __restrict__ cross_list,
+                       float* __restrict__ partial) {
   constexpr int VI = (Vec<TIn>::N > Vec<TOut>::N) ? Vec<TIn>::N : Vec<TOut>::N;
+  constexpr int LD = VI / Vec<TIn>::N;  // 16-byte loads per row per thread
+  __shared__ int s_off[kSegBlk + 1];    // offsets of the segments that can touch this block
   __shared__ int s_row[kSegBlk];
-  __shared__ int s_seg[kSegBlk];
-  __shared__ int s_seg_begin[kSegBlk];
-  __shared__ int s_seg_end[kSegBlk];
+  __shared__ int s_loc[kSegBlk];        // position -> index into s_off
   const int blk = blockIdx.x;
   const int p0 = blk * kSegBlk;
   const int cnt = min(kSegBlk, T - p0);
   const int n_u = *n_unique;
+
+  // r_first = largest r with seg_offsets[r] <= p0, found with kThreads pivots per round
+  // (two rounds for a few thousand segments instead of a dozen dependent loads).
+  int lo = 0, hi = n_u;  // seg_offsets[lo] <= p0 < seg_offsets[hi]
+  while (hi - lo > 1) {
+    const int step = (hi - lo + kThreads) / (kThreads + 1);
+    const int piv = lo + (static_cast<int>(threadIdx.x) + 1) * step;
+    const int hit = (piv < hi && seg_offsets[piv] <= p0) ? 1 : 0;
+    const int n_hit = __syncthreads_count(hit);
+    const int new_lo = lo + n_hit * step;
+    hi = min(hi, new_lo + step);
+    lo = new_lo;
+  }
+  const int r_first = lo;
+  if (threadIdx.x <= kSegBlk) {
+    const int r = r_first + threadIdx.x;
+    s_off[threadIdx.x] = r <= n_u ? seg_offsets[r] : 0x7fffffff;
+  }
+  if (threadIdx.x < cnt) s_row[threadIdx.x] = perm[p0 + threadIdx.x];
+  __syncthreads();
   if (threadIdx.x < cnt) {
     const int p = p0 + threadIdx.x;
-    const int r = segment_of(seg_offsets, n_u, p);
-    s_row[threadIdx.x] = perm[p];
-    s_seg[threadIdx.x] = r;
-    s_seg_begin[threadIdx.x] = seg_offsets[r];
-    s_seg_end[threadIdx.x] = seg_offsets[r + 1];
+    int a = 0, b = kSegBlk;  // s_off[a] <= p; at most kSegBlk segments start inside the block
+    while (b - a > 1) {
+      const int mid = (a + b) >> 1;
+      if (s_off[mid] <= p) a = mid; else b = mid;
+    }
+    if (s_off[b] <= p) a = b;
+    s_loc[threadIdx.x] = a;
   }
   __syncthreads();
+  if (blockIdx.y == 0 && threadIdx.x == 0) {
+    // a segment that starts in this block and runs past its end is finished by pass 2
+    const int j = s_loc[cnt - 1];
+    if (s_off[j] >= p0 && s_off[j + 1] > p0 + kSegBlk) cross_list[1 + atomicAdd(cross_list, 1)] = blk;
+  }
   const int col = (blockIdx.y * kThreads + threadIdx.x) * VI;
   if (col >= F) return;
 
@@ -103,20 +127,14 @@ segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* 
 #pragma unroll
   for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
   bool first_run = true;
-
   for (int b0 = 0; b0 < cnt; b0 += kBatch) {
-    float v[kBatch][VI];
+    uint4 raw[kBatch][LD];
 #pragma unroll
     for (int j = 0; j < kBatch; ++j) {
       if (b0 + j < cnt) {
         const TIn* src = dU + static_cast<size_t>(s_row[b0 + j]) * F + col;
 #pragma unroll
-        for (int i = 0; i < VI; i += Vec<TIn>::N) {
-          float t[Vec<TIn>::N];
-          Vec<TIn>::load(src + i, t);
-#pragma unroll
-          for (int q = 0; q < Vec<TIn>::N; ++q) v[j][i + q] = t[q];
-        }
+        for (int i = 0; i < LD; ++i) raw[j][i] = Vec<TIn>::load_raw(src + i * Vec<TIn>::N);
       }
     }
 #pragma unroll
@@ -124,15 +142,15 @@ segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* 
       const int q = b0 + j;
       if (q < cnt) {
 #pragma unroll
-        for (int i = 0; i < VI; ++i) acc[i] += v[j][i];
-        const bool run_ends = (q + 1 == cnt) || (s_seg[q + 1] != s_seg[q]);
+        for (int i = 0; i < LD; ++i) Vec<TIn>::add(acc + i * Vec<TIn>::N, raw[j][i]);
+        const int loc = s_loc[q];
+        const bool run_ends = (q + 1 == cnt) || (s_loc[q + 1] != loc);
         if (run_ends) {
-          const bool whole = s_seg_begin[q] >= p0 && s_seg_end[q] <= p0 + kSegBlk;
+          const bool whole = s_off[loc] >= p0 && s_off[loc + 1] <= p0 + kSegBlk;
           if (whole) {
-            store_row<VI, TOut>(dE_rows + static_cast<size_t>(s_seg[q]) * F + col, acc);
+            store_row<VI, TOut>(dE_rows + static_cast<size_t>(r_first + loc) * F + col, acc);
           } else {
-            float* dst = partial + (static_cast<size_t>(2 * blk + (first_run ? 0 : 1))) * F + col;
-            store_row<VI, float>(dst, acc);
+            store_row<VI, float>(partial + static_cast<size_t>(2 * blk + (first_run ? 0 : 1)) * F + col, acc);
           }
 #pragma unroll
           for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
@@ -143,38 +161,64 @@ segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* 
   }
 }
 
+// One CTA per (crossing segment, 32 x VI columns): kRowLanes partial rows are added side by
+// side, each lane walking its rows in block order, then the lanes are combined in lane order.
 template <typename TOut, int VI>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kRowLanes * kColLanes, 4)
 segreduce_pass2_kernel(int T, int F, const int32_t* __restrict__ seg_offsets,
-                       const int32_t* __restrict__ n_unique, const float* __restrict__ partial,
-                       TOut* __restrict__ dE_rows) {
-  const int blk = blockIdx.x;
-  const int p0 = blk * kSegBlk;
-  const int p_last = min(T, p0 + kSegBlk) - 1;
+                       const int32_t* __restrict__ n_unique, const int32_t* __restrict__ cross_list,
+                       const float* __restrict__ partial, TOut* __restrict__ dE_rows) {
+  __shared__ float s_sum[kRowLanes][kColLanes][VI + 1];
+  __shared__ int s_r;
+  const int n_cross = cross_list[0];
   const int n_u = *n_unique;
-  // the segment of this block's last position; this CTA owns it iff it starts here and
-  // runs past the block's end
-  const int r = segment_of(seg_offsets, n_u, p_last);
-  const int seg_begin = seg_offsets[r], seg_end = seg_offsets[r + 1];
-  if (seg_begin < p0 || seg_end <= p0 + kSegBlk) return;
-  const int col = (blockIdx.y * kThreads + threadIdx.x) * VI;
-  if (col >= F) return;
-  const int b_last = (seg_end - 1) / kSegBlk;
-  float acc[VI];
-#pragma unroll
-  for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
-  for (int b = blk; b <= b_last; ++b) {
-    // the segment's run is the first run of block b unless b is the starting block and the
-    // segment does not begin exactly at the block's first position
-    const int slot = (b > blk || seg_begin == p0) ? 2 * b : 2 * b + 1;
-    const float* src = partial + static_cast<size_t>(slot) * F + col;
-#pragma unroll
-    for (int i = 0; i < VI; i += 4) {
-      const float4 q = *reinterpret_cast<const float4*>(src + i);
-      acc[i] += q.x; acc[i + 1] += q.y; acc[i + 2] += q.z; acc[i + 3] += q.w;
+  const int cl = threadIdx.x % kColLanes, rl = threadIdx.x / kColLanes;
+  const int col = (blockIdx.y * kColLanes + cl) * VI;
+  for (int e = blockIdx.x; e < n_cross; e += gridDim.x) {
+    const int blk = cross_list[1 + e];
+    const int p0 = blk * kSegBlk;
+    if (threadIdx.x == 0) {
+      // the segment of the block's last position
+      const int p_last = min(T, p0 + kSegBlk) - 1;
+      int lo = 0, hi = n_u;
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (seg_offsets[mid] <= p_last) lo = mid; else hi = mid;
+      }
+      s_r = lo;
     }
+    __syncthreads();
+    const int r = s_r;
+    const int seg_begin = seg_offsets[r], seg_end = seg_offsets[r + 1];
+    const int b_last = (seg_end - 1) / kSegBlk;
+    float acc[VI];
+#pragma unroll
+    for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
+    if (col < F) {
+      for (int b = blk + rl; b <= b_last; b += kRowLanes) {
+        // the segment's run is the first run of block b, unless b is the block it starts in
+        // and it does not start at that block's first position
+        const int slot = (b > blk || seg_begin == p0) ? 2 * b : 2 * b + 1;
+        const float* src = partial + static_cast<size_t>(slot) * F + col;
+#pragma unroll
+        for (int i = 0; i < VI; i += 4) {
+          const float4 q = *reinterpret_cast<const float4*>(src + i);
+          acc[i] += q.x; acc[i + 1] += q.y; acc[i + 2] += q.z; acc[i + 3] += q.w;
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < VI; ++i) s_sum[rl][cl][i] = acc[i];
+    __syncthreads();
+    if (rl == 0 && col < F) {
+#pragma unroll
+      for (int l = 1; l < kRowLanes; ++l)
+#pragma unroll
+        for (int i = 0; i < VI; ++i) acc[i] += s_sum[l][cl][i];
+      store_row<VI, TOut>(dE_rows + static_cast<size_t>(r) * F + col, acc);
+    }
+    __syncthreads();
   }
-  store_row<VI, TOut>(dE_rows + static_cast<size_t>(r) * F + col, acc);
 }
 
 template <typename TIn, typename TOut>
@@ -182,12 +226,17 @@ cudaError_t launch_typed(int T, int F, const void* dU, const int32_t* perm, cons
                          const int32_t* n_unique, void* dE_rows, void* scratch, cudaStream_t stream) {
   constexpr int VI = (Vec<TIn>::N > Vec<TOut>::N) ? Vec<TIn>::N : Vec<TOut>::N;
   const int n_blk = (T + kSegBlk - 1) / kSegBlk;
-  dim3 grid(n_blk, (F + kThreads * VI - 1) / (kThreads * VI));
-  segreduce_pass1_kernel<TIn, TOut><<<grid, kThreads, 0, stream>>>(
-      T, F, static_cast<const TIn*>(dU), perm, seg_offsets, n_unique, static_cast<TOut*>(dE_rows),
-      static_cast<float*>(scratch));
-  segreduce_pass2_kernel<TOut, VI><<<grid, kThreads, 0, stream>>>(
-      T, F, seg_offsets, n_unique, static_cast<const float*>(scratch), static_cast<TOut*>(dE_rows));
+  int32_t* cross_list = static_cast<int32_t*>(scratch);
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(scratch) + partial_offset_bytes(n_blk));
+  cudaError_t e = cudaMemsetAsync(cross_list, 0, sizeof(int32_t), stream);
+  if (e != cudaSuccess) return e;
+  dim3 grid1(n_blk, (F + kThreads * VI - 1) / (kThreads * VI));
+  segreduce_pass1_kernel<TIn, TOut><<<grid1, kThreads, 0, stream>>>(
+      T, F, static_cast<const TIn*>(dU), perm, seg_offsets, n_unique, static_cast<TOut*>(dE_rows), cross_list,
+      partial);
+  dim3 grid2(n_blk < 64 ? n_blk : 64, (F + kColLanes * VI - 1) / (kColLanes * VI));
+  segreduce_pass2_kernel<TOut, VI><<<grid2, kRowLanes * kColLanes, 0, stream>>>(
+      T, F, seg_offsets, n_unique, cross_list, partial, static_cast<TOut*>(dE_rows));
   count_launches(2);
   return cudaGetLastError();
 }
@@ -197,7 +246,7 @@ cudaError_t launch_typed(int T, int F, const void* dU, const int32_t* perm, cons
 size_t segreduce_workspace_bytes(int T, int F) {
   if (T <= 0) return 0;
   const size_t n_blk = (static_cast<size_t>(T) + kSegBlk - 1) / kSegBlk;
-  return align_up(2 * n_blk * static_cast<size_t>(F) * sizeof(float), 256);
+  return partial_offset_bytes(static_cast<int>(n_blk)) + align_up(2 * n_blk * static_cast<size_t>(F) * sizeof(float), 256);
 }
 
 cudaError_t launch_segreduce(int T, int F, int in_dtype, int out_dtype, const void* dU,
