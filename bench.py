@@ -41,12 +41,29 @@ def load_peaks():
     return dict(FALLBACK_PEAKS, source="fallback")
 
 
-def load_traffic(workload: str):
-    p = os.path.join(ROOT, "profiles", "ncu_traffic.json")
-    if os.path.exists(p):
-        with open(p) as f:
-            return json.load(f).get(workload, {})
-    return {}
+def source_digest(files) -> str:
+    """Short digest of kernel sources: ties stored DRAM counters to the code they were taken from."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in files:
+        with open(os.path.join(ROOT, "paper_2601_10639_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+def load_traffic(step: str):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture) of the
+    kernel behind `step`, scaled to this workload's launch; None when no capture is stored or the
+    kernel's source has changed since it was taken.  File lines: step tokens_captured bytes digest."""
+    p = os.path.join(ROOT, "profiles", "ncu_traffic.txt")
+    if not os.path.exists(p):
+        return None
+    digest = source_digest(["gemm_sm100.cu", "ptx_sm100.cuh"] if step.endswith("_gemm") else ["segreduce.cu"])
+    for line in open(p):
+        parts = line.split()
+        if len(parts) >= 4 and not line.startswith("#") and parts[0] == step and parts[3] == digest:
+            return int(parts[1]), float(parts[2])
+    return None
 
 
 class ClockSampler:
@@ -152,13 +169,16 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="stem", choices=["stem", "reference"])
     ap.add_argument("--workload", default="1b", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--cpu-tokens", type=int, default=8192, help="tokens in the CPU-baseline sample (0 = skip)")
     ap.add_argument("--ref-tokens", type=int, default=1024, help="tokens per step of --impl reference")
     ap.add_argument("--seed", type=int, default=synth.BASE_SEED)
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="override the workload's token count (small cases for profiler captures; not a bench line)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.warmup < 3:
@@ -186,7 +206,7 @@ def main():
 
     dcode = B.DTYPE_BF16 if w.dtype == "bf16" else B.DTYPE_FP32
     dt = runner.torch_dtype(dcode)
-    T, d, F, V = w.T, w.d_model, w.d_ff, w.V
+    T, d, F, V = (args.tokens or w.T), w.d_model, w.d_ff, w.V
     backward = w.backward
     # ---- synthetic inputs (every rank its own batch; same shapes) -----------------------
     gen = torch.Generator(device=dev).manual_seed(args.seed + 1000 * rank)
@@ -237,7 +257,7 @@ def main():
     # ---- end to end through the host-buffer entry point -------------------------------------
     esz = 2 if dcode == B.DTYPE_BF16 else 4
     e2e = None
-    if backward:
+    if backward and not args.no_e2e:
         hx, hdy = st.x.cpu().pin_memory(), st.dy.cpu().pin_memory()
         hids = st.ids.cpu().pin_memory()
         hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
@@ -301,14 +321,17 @@ def main():
             k["frac_of_measured_hbm"] = k["gbs"] / peaks["hbm_gbs"]
         kernels[name] = k
     gemms = {n: k for n, k in kernels.items() if n.endswith("_gemm")}
-    traffic = load_traffic(w.name)
     roofline = None
     if gemms and dcode == B.DTYPE_BF16:
         dom = max(gemms, key=lambda n: gemms[n]["avg_ms"])
+        cap = load_traffic(dom)
+        # DRAM traffic grows in proportion to the tokens of a launch (every [T,.] operand does; the
+        # weights are the small remainder), so a capture at fewer tokens is scaled by T / T_captured.
+        traffic = cap[1] * T / cap[0] if cap else None
         roofline = {"kernel": dom, "bound": "tensor", "achieved": gemms[dom]["tflops"],
                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                     "frac": gemms[dom]["tflops"] / peaks["bf16_tflops_sustained"],
-                    "traffic": traffic.get(dom), "peak_source": peaks["source"] + " (sustained bf16 GEMM)",
+                    "traffic": traffic, "peak_source": peaks["source"] + " (sustained bf16 GEMM, of measured)",
                     "flops_per_launch": flops_gemm}
 
     # ---- the CPU checker timed beside it (rank 0, N = 1 only) -----------------------------------------

@@ -86,7 +86,7 @@ int stem_init_workspace(void* ws, size_t ws_bytes, void* stream);
 int stem_query_status(const void* ws, void* stream, int32_t* status_out /*host*/);
 
 /*
- * Token deduplication (Section 3.3 "System Implementation": the batch's token ids are
+ * Token deduplication (Section 3.4 "System Implementation": the batch's token ids are
  * deduplicated so only uniq(B*L) rows move; Table 1, "Communication").  The paper
  * names the step; the arrays are defined here, each with exactly one correct value:
  *   perm[T]          positions sorted by (ids[t], t) ascending (stable radix sort by id)
@@ -160,7 +160,7 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
                       void* stream);
 
 /*
- * Row prefetch for a table kept off the device (Section 3.3: tables offloaded to CPU
+ * Row prefetch for a table kept off the device (Section 3.4: tables offloaded to CPU
  * memory, rows of the deduplicated ids prefetched asynchronously with layer compute;
  * Figure 1(c)):   dev_cache[r,:] = table[ids[r],:]   for r < *n_ids.
  * table: [V,d_ff] (dtype) in page-locked host memory (cudaHostAlloc / cudaHostRegister;
@@ -199,7 +199,7 @@ int stem_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t a_mn,
 
 /*
  * One training step of the layer from host buffers (the composition of the calls above,
- * in the order Section 3.3 gives for training: ids deduplicated, forward, backward, table
+ * in the order Section 3.4 gives for training: ids deduplicated, forward, backward, table
  * gradients reduced per unique id):
  *   copy host_x, host_ids, host_dy to the device; stem_dedup_ids; stem_ffn_forward;
  *   stem_ffn_backward; copy y and dx back to host_y, host_dx (and n_u to host_n_unique

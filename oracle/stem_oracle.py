@@ -12,7 +12,7 @@ It is deliberately unblocked and unfused so it can be read against the equations
 * backward  -- the paper gives no formulas (it only says training sends the table's
               gradients back, Table 1 notes); these are the chain rule of the forward
               for the loss  L = sum_{t,i} dy[t,i] * y[t,i].
-* dedup     -- the paper only names token deduplication (Section 3.3); the arrays are
+* dedup     -- the paper only names token deduplication (Section 3.4); the arrays are
               defined here: positions stably sorted by id, the distinct ids ascending,
               where each id's run starts, and each position's slot.
 
@@ -65,7 +65,7 @@ def forward(x, ids, W_gate, E, W_down, return_intermediates: bool = False):
 
 
 def dedup(ids):
-    """Index arrays of token deduplication (Section 3.3 names the step only).
+    """Index arrays of token deduplication (Section 3.4 names the step only).
 
     perm        : positions sorted by (ids[t], t) ascending  -- a stable sort by id
     unique_ids  : the distinct ids, ascending
@@ -133,7 +133,7 @@ def dE_dense(unique_ids, dE_rows, V: int) -> np.ndarray:
 
 
 def prefetch_rows(unique_ids, n_ids: int, host_E) -> np.ndarray:
-    """Row cache of the offloaded-table path (Section 3.3; Figure 1(c)):
+    """Row cache of the offloaded-table path (Section 3.4; Figure 1(c)):
     cache[r] = E[unique_ids[r]] for r < n_ids."""
     idx = np.asarray(unique_ids[:n_ids], dtype=np.int64)
     return np.asarray(host_E)[idx].copy()

@@ -13,8 +13,8 @@ Distributions follow the layer's workloads: activations and upstream
 gradients ~ N(0, 1); W_gate ~ N(0, 1/d_model); W_down ~ N(0, 1/d_ff);
 E ~ N(0, 0.02^2); token ids uniform, Zipf(s) with P(id = k) ~ (k + 1)^-s, or a
 per-position Bernoulli mix of the two (Zipfian token frequencies: paper
-Section 2 "Unbalanced expert frequency" and Section 3.3 "System
-Implementation"; sublinear unique-token growth: Section 3.2.3).
+Section 2 "Unbalanced expert frequency" and Section 3.4 "System
+Implementation"; sublinear unique-token growth: Section 3.2.5).
 """
 from __future__ import annotations
 
