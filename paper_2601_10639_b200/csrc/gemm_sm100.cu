@@ -10,9 +10,13 @@
 //               instruction, four per 64-wide k block) and commits to mbarriers
 //   warps 2..9  epilogue: tcgen05.ld the finished 128 x BN fp32 tile (one row per thread,
 //               two warps per TMEM lane quarter, each taking half of the columns), apply
-//               the fused elementwise step, store.  The table row and the saved G are
-//               fetched one 32-column chunk ahead of the arithmetic, with 32-byte
-//               accesses, so their latency hides behind the previous chunk
+//               the fused elementwise step, and hand the result to TMA: each warp writes a
+//               32-row x 32-column block into its own swizzled shared-memory buffer and
+//               one lane issues a tensor store, so global writes are whole lines issued
+//               by the copy engine instead of 32 scattered sectors per instruction.  The
+//               table row and the saved G are fetched one 32-column chunk ahead of the
+//               arithmetic, with 32-byte loads, so their latency hides behind the
+//               previous chunk
 // Two accumulator tiles live in TMEM (2 x BN columns), so the epilogue of tile i overlaps
 // the MMAs of tile i+1.  Operands may be K-major or MN-major (the backward pass contracts
 // over the token dimension, which is the slow index of every [T, .] tensor); both use the
@@ -42,7 +46,10 @@ struct Smem {
   static constexpr int kABytes = BM * BK * 2;
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kBarOffset = STAGES * kStageBytes;
+  // per epilogue warp: two 2 KB output blocks (32 rows x 32 bf16) or one 4 KB block (fp32)
+  static constexpr int kOutOffset = STAGES * kStageBytes;
+  static constexpr int kOutBytesPerWarp = 4096;
+  static constexpr int kBarOffset = kOutOffset + kEpiWarps * kOutBytesPerWarp;
   // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain, tmem address, abort
   static constexpr int kNumBars = 2 * STAGES + 5;
   static constexpr int kTotal = kBarOffset + kNumBars * 8 + 16 + 1024;  // + alignment slack
@@ -60,17 +67,9 @@ __device__ __forceinline__ void ldg256(const void* p, uint32_t* r) {
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                : "l"(p));
 }
-__device__ __forceinline__ void stg256(void* p, const uint32_t* r) {
-  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
-               ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-               : "memory");
-}
 __device__ __forceinline__ void ldg128(const void* p, uint32_t* r) {
   const uint4 q = __ldg(static_cast<const uint4*>(p));
   r[0] = q.x; r[1] = q.y; r[2] = q.z; r[3] = q.w;
-}
-__device__ __forceinline__ void stg128(void* p, const uint32_t* r) {
-  *static_cast<uint4*>(p) = make_uint4(r[0], r[1], r[2], r[3]);
 }
 
 // 32 bf16 (16 registers) starting at column n of a row; p points at column n.
@@ -84,26 +83,6 @@ __device__ __forceinline__ void load_bf16x32(const __nv_bfloat16* p, int n, int 
     for (int q = 0; q < 4; ++q) if (n + 8 * q < N) ldg128(p + 8 * q, r + 4 * q);
   }
 }
-template <bool WIDE>
-__device__ __forceinline__ void store_bf16x32(__nv_bfloat16* p, int n, int N, const uint32_t (&r)[16]) {
-  if (WIDE) {
-#pragma unroll
-    for (int h = 0; h < 2; ++h) if (n + 16 * h < N) stg256(p + 16 * h, r + 8 * h);
-  } else {
-#pragma unroll
-    for (int q = 0; q < 4; ++q) if (n + 8 * q < N) stg128(p + 8 * q, r + 4 * q);
-  }
-}
-template <bool WIDE>
-__device__ __forceinline__ void store_f32x32(float* p, int n, int N, const uint32_t (&r)[32]) {
-  if (WIDE) {
-#pragma unroll
-    for (int h = 0; h < 4; ++h) if (n + 8 * h < N) stg256(p + 8 * h, r + 8 * h);
-  } else {
-#pragma unroll
-    for (int q = 0; q < 8; ++q) if (n + 4 * q < N) stg128(p + 4 * q, r + 4 * q);
-  }
-}
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -111,20 +90,38 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// Fused elementwise step on 32 consecutive columns of one output row.  e and g hold the
+// One row (lane) of a 32-row block into the warp's staging buffer, in the layout the
+// output tensor maps expect.  bf16: 64-byte rows, 64-byte swizzle (16-byte piece j of row
+// r sits at piece j ^ ((r >> 1) & 3)).  fp32: 128-byte rows, 128-byte swizzle (piece j at
+// j ^ (r & 7)).  Both patterns are bank-conflict free for 16-byte stores by 8 lanes.
+__device__ __forceinline__ void stage_row_bf16(uint32_t buf, int lane, const uint32_t (&o)[16]) {
+  const uint32_t row = buf + lane * 64, x = (lane >> 1) & 3;
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    ptx::st_shared_v4(row + ((j ^ x) << 4), o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+}
+__device__ __forceinline__ void stage_row_f32(uint32_t buf, int lane, const uint32_t (&o)[32]) {
+  const uint32_t row = buf + lane * 128, x = lane & 7;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    ptx::st_shared_v4(row + ((j ^ x) << 4), o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+}
+
+// Fused elementwise step on 32 consecutive columns of one output row: results go to the
+// warp's staging buffer (first output at buf, second at buf + 2048).  e and g hold the
 // table row segment and the saved pre-activation (bf16 pairs), fetched earlier.
-template <int KIND, bool WIDE>
-__device__ __forceinline__ void epilogue_row32(const EpiParams& ep, size_t off, int n, int N,
+template <int KIND>
+__device__ __forceinline__ void epilogue_row32(const EpiParams& ep, uint32_t buf, int lane,
                                                const uint32_t (&acc)[32], const uint32_t (&e)[16],
                                                const uint32_t (&g)[16]) {
   if (KIND == kEpiStore) {
     if (ep.out_fp32) {
-      store_f32x32<WIDE>(static_cast<float*>(ep.out) + off, n, N, acc);
+      stage_row_f32(buf, lane, acc);
     } else {
       uint32_t o[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
-      store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.out) + off, n, N, o);
+      stage_row_bf16(buf, lane, o);
     }
   } else if (KIND == kEpiGate) {
     uint32_t h[16], go[16];
@@ -134,8 +131,8 @@ __device__ __forceinline__ void epilogue_row32(const EpiParams& ep, size_t off, 
       h[i] = pack_bf16(a0 * fast_sigmoid(a0) * bf16_lo(e[i]), a1 * fast_sigmoid(a1) * bf16_hi(e[i]));
       go[i] = pack_bf16(a0, a1);
     }
-    store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.H) + off, n, N, h);
-    if (ep.G) store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.G) + off, n, N, go);
+    stage_row_bf16(buf, lane, h);
+    if (ep.G) stage_row_bf16(buf + 2048, lane, go);
   } else {
     uint32_t du[16], dg[16];
 #pragma unroll
@@ -147,8 +144,8 @@ __device__ __forceinline__ void epilogue_row32(const EpiParams& ep, size_t off, 
       dg[i] = pack_bf16(a0 * bf16_lo(e[i]) * (s0 * (1.0f + g0 * (1.0f - s0))),
                         a1 * bf16_hi(e[i]) * (s1 * (1.0f + g1 * (1.0f - s1))));
     }
-    store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.H) + off, n, N, du);
-    store_bf16x32<WIDE>(static_cast<__nv_bfloat16*>(ep.G) + off, n, N, dg);
+    stage_row_bf16(buf, lane, du);
+    stage_row_bf16(buf + 2048, lane, dg);
   }
 }
 
@@ -165,6 +162,7 @@ __device__ __forceinline__ TileCoord tile_coord(int tile, int tiles_m, int tiles
 template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                int M, int N, int K, int group_m, EpiParams ep) {
   using L = Smem<BN, STAGES>;
   extern __shared__ uint8_t smem_raw[];
@@ -194,6 +192,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
+    ptx::prefetch_tensormap(&tmC0);
+    if (KIND != kEpiStore) ptx::prefetch_tensormap(&tmC1);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
@@ -289,11 +289,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;       // which half of the tile's columns it handles
     constexpr int kChunks = BN / 2 / 32;    // 32-column chunks per thread per tile
+    const uint32_t out_buf = base + L::kOutOffset + (warp - 2) * L::kOutBytesPerWarp;
+    const bool second_out = KIND == kEpiDH || (KIND == kEpiGate && ep.G != nullptr);
     int acc = 0; uint32_t aph = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       const TileCoord tc = tile_coord(tile, tiles_m, tiles_n, group_m);
-      const int m = tc.m_blk * BM + q * 32 + lane;
+      const int m_warp = tc.m_blk * BM + q * 32;  // first row of this warp's 32-row block
+      const int m = m_warp + lane;
       const int n0 = tc.n_blk * BN + half * (BN / 2);
       const bool row_ok = m < M;
       const size_t row_off = static_cast<size_t>(m) * N;
@@ -335,13 +338,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint32_t v[32];
         ptx::tmem_ld_32x32(t_row + c * 32, v);
         ptx::tmem_ld_wait();
-        if (row_ok) epilogue_row32<KIND, WIDE>(ep, row_off + n, n, N, v, e_cur, g_cur);
+        if (c + 1 == kChunks) {
+          // the accumulator has been read out: hand it back to the MMA issuer
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+        }
+        // the staging buffer is free once the previous chunk's tensor stores have read it
+        if (lane == 0) ptx::bulk_wait_read_all();
+        __syncwarp();
+        epilogue_row32<KIND>(ep, out_buf, lane, v, e_cur, g_cur);
+        ptx::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0 && m_warp < M && n < N) {
+          ptx::tma_store_2d(&tmC0, out_buf, n, m_warp);
+          if (second_out) ptx::tma_store_2d(&tmC1, out_buf + 2048, n, m_warp);
+          ptx::bulk_commit_group();
+        }
       }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; aph ^= 1u; }
     }
+    // every tensor store of this warp must be complete before the CTA may exit
+    if (lane == 0) ptx::bulk_wait_all();
   }
 
   __syncthreads();
@@ -393,9 +411,26 @@ bool encode_map(CUtensorMap* map, const void* ptr, int rows, int cols, int box_r
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Output matrix [rows, cols] row-major, bf16 or fp32; box = 32 columns x 32 rows, swizzled
+// over the box's row length (64 bytes for bf16, 128 bytes for fp32).
+bool encode_out_map(CUtensorMap* map, const void* ptr, int rows, int cols, bool fp32) {
+  EncodeFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t esz = fp32 ? 4 : 2;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * esz};
+  const cuuint32_t box[2] = {32u, 32u};
+  const cuuint32_t estr[2] = {1u, 1u};
+  return fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            fp32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE>
-cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, int M, int N, int K,
-                        const EpiParams& ep, cudaStream_t stream) {
+cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC0,
+                        const CUtensorMap& tmC1, int M, int N, int K, const EpiParams& ep,
+                        cudaStream_t stream) {
   using L = Smem<BN, STAGES>;
   auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES, WIDE>;
   static bool configured = false;
@@ -406,7 +441,7 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, int M, i
   }
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = tiles < device_sm_count() ? tiles : device_sm_count();
-  kern<<<grid, kThreads, L::kTotal, stream>>>(tmA, tmB, M, N, K, 8, ep);
+    kern<<<grid, kThreads, L::kTotal, stream>>>(tmA, tmB, tmC0, tmC1, M, N, K, 8, ep);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -419,10 +454,20 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
   const bool okA = A_MN ? encode_map(&tmA, A, K, M, BK) : encode_map(&tmA, A, M, K, BM);
   const bool okB = B_MN ? encode_map(&tmB, B, K, N, BK) : encode_map(&tmB, B, N, K, BN);
   if (!okA || !okB) return cudaErrorNotSupported;
+  CUtensorMap tmC0, tmC1;
+  bool okC;
+  if (KIND == kEpiStore) {
+    okC = encode_out_map(&tmC0, ep.out, M, N, ep.out_fp32 != 0);
+    tmC1 = tmC0;
+  } else {
+    okC = encode_out_map(&tmC0, ep.H, M, N, false);
+    if (ep.G) okC = okC && encode_out_map(&tmC1, ep.G, M, N, false); else tmC1 = tmC0;
+  }
+  if (!okC) return cudaErrorNotSupported;
   auto a32 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; };
-  const bool wide = (N % 16 == 0) && a32(ep.out) && a32(ep.E) && a32(ep.H) && a32(ep.G) && a32(ep.Gin);
-  if (wide) return launch_inst<A_MN, B_MN, KIND, BN, STAGES, true>(tmA, tmB, M, N, K, ep, stream);
-  return launch_inst<A_MN, B_MN, KIND, BN, STAGES, false>(tmA, tmB, M, N, K, ep, stream);
+  const bool wide = (N % 16 == 0) && a32(ep.E) && a32(ep.Gin);
+  if (wide) return launch_inst<A_MN, B_MN, KIND, BN, STAGES, true>(tmA, tmB, tmC0, tmC1, M, N, K, ep, stream);
+  return launch_inst<A_MN, B_MN, KIND, BN, STAGES, false>(tmA, tmB, tmC0, tmC1, M, N, K, ep, stream);
 }
 
 }  // namespace
