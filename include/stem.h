@@ -55,6 +55,7 @@ extern "C" {
 #define STEM_DTYPE_BF16 1
 
 #define STEM_FLAG_SIMT 1 /* run the bf16 contractions on the plain-FMA kernels (debug aid) */
+#define STEM_FLAG_SINGLE_CTA 2 /* tensor-core contractions on single CTAs instead of CTA pairs (debug aid) */
 
 typedef struct {
   int32_t T;          /* positions in this call (batch x sequence)                 */

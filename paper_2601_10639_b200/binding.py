@@ -23,6 +23,7 @@ ERR_WORKSPACE_TOO_SMALL, ERR_NOT_PINNED, ERR_CUDA, ERR_TIMEOUT, ERR_ID_RANGE = -
 ERR_STATIC_LIMIT = -9
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 FLAG_SIMT = 1
+FLAG_SINGLE_CTA = 2
 
 EXPORTS = (
     "stem_version", "stem_status_string", "stem_workspace_bytes", "stem_init_workspace",

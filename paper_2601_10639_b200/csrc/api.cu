@@ -129,7 +129,7 @@ bool use_tc(const stem_shape_t* s) {
 
 cudaError_t gemm(const stem_shape_t* s, int M, int N, int K, const void* A, bool a_mn, const void* B,
                  bool b_mn, EpiKind kind, const EpiParams& ep, cudaStream_t st) {
-  if (use_tc(s)) return launch_tc_gemm(M, N, K, A, a_mn, B, b_mn, kind, ep, st);
+  if (use_tc(s)) return launch_tc_gemm(M, N, K, A, a_mn, B, b_mn, kind, ep, !(s->flags & STEM_FLAG_SINGLE_CTA), st);
   return launch_simt_gemm(s->dtype, M, N, K, A, a_mn, B, b_mn, kind, ep, st);
 }
 
@@ -347,7 +347,8 @@ int stem_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t a_mn,
     e = launch_simt_gemm(STEM_DTYPE_BF16, M, N, K, A, a_mn != 0, B, b_mn != 0, kEpiStore, p, static_cast<cudaStream_t>(stream));
   } else {
     if (!is_sm100()) return STEM_ERR_UNSUPPORTED_ARCH;
-    e = launch_tc_gemm(M, N, K, A, a_mn != 0, B, b_mn != 0, kEpiStore, p, static_cast<cudaStream_t>(stream));
+    e = launch_tc_gemm(M, N, K, A, a_mn != 0, B, b_mn != 0, kEpiStore, p, !(flags & STEM_FLAG_SINGLE_CTA),
+                       static_cast<cudaStream_t>(stream));
   }
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
 }

@@ -41,10 +41,13 @@ constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr long long kWaitLimitCycles = 2000000000ll;  // ~1 s at boost clock
 constexpr int kAtomBytes = 64 * BK * 2;                // one 64(MN) x BK swizzled block
 
-template <int BN, int STAGES>
+// CTAS = 2: two CTAs of a cluster share every MMA (cta_group::2).  Each stages its own 128
+// rows of A and half of the BN columns of B, so a stage is 32 KB instead of 48 KB and the
+// operand bytes fetched per flop drop by a third.
+template <int BN, int STAGES, int CTAS>
 struct Smem {
   static constexpr int kABytes = BM * BK * 2;
-  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kBBytes = (BN / CTAS) * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   // per epilogue warp: two 2 KB output blocks (32 rows x 32 bf16) or one 4 KB block (fp32)
   static constexpr int kOutOffset = STAGES * kStageBytes;
@@ -159,12 +162,12 @@ __device__ __forceinline__ TileCoord tile_coord(int tile, int tiles_m, int tiles
   return {first_m + in % gsize, in / gsize};
 }
 
-template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE>
+template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                int M, int N, int K, int group_m, EpiParams ep) {
-  using L = Smem<BN, STAGES>;
+  using L = Smem<BN, STAGES, CTAS>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -179,14 +182,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kBarOffset + L::kNumBars * 8 + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
+  // A work unit is one BM*CTAS x BN output tile, handled by one CTA or one CTA pair.
+  const uint32_t rank = CTAS == 2 ? ptx::cluster_ctarank() : 0u;
+  const int unit0 = blockIdx.x / CTAS, unit_stride = gridDim.x / CTAS;
+  const int tiles_m = (M + BM * CTAS - 1) / (BM * CTAS), tiles_n = (N + BN - 1) / BN;
   const int num_tiles = tiles_m * tiles_n;
   const int k_blocks = (K + BK - 1) / BK;
   constexpr uint32_t kTmemCols = 2 * BN;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { ptx::mbar_init(tfull_bar(a), 1); ptx::mbar_init(tempty_bar(a), kEpiWarps); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(tfull_bar(a), 1); ptx::mbar_init(tempty_bar(a), kEpiWarps * CTAS); }
     ptx::mbar_init(drain_bar, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
@@ -196,11 +202,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (KIND != kEpiStore) ptx::prefetch_tensormap(&tmC1);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
-    ptx::tmem_relinquish();
+    if (CTAS == 2) {
+      ptx::tmem_alloc_pair(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+      ptx::tmem_relinquish_pair();
+    } else {
+      ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before();
-  __syncthreads();
+  // in a pair, the other CTA's barriers and TMEM must exist before anything targets them
+  if (CTAS == 2) ptx::cluster_sync(); else __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -210,9 +222,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) {
       int s = 0; uint32_t ph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int tile = unit0; tile < num_tiles && ok; tile += unit_stride) {
         const TileCoord tc = tile_coord(tile, tiles_m, tiles_n, group_m);
-        const int m0 = tc.m_blk * BM, n0 = tc.n_blk * BN;
+        // this CTA's rows of A and its share of the columns of B
+        const int m0 = (tc.m_blk * CTAS + rank) * BM, n0 = tc.n_blk * BN + rank * (BN / CTAS);
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitCycles)) {
             report_error(ep.status, STEM_ERR_TIMEOUT, 1);
@@ -220,19 +233,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
           const uint32_t a_dst = base + s * L::kStageBytes;
           const uint32_t b_dst = a_dst + L::kABytes;
-          ptx::mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
+          // The MMA issuer (rank 0) waits on its own full barrier for the bytes of both CTAs.
+          if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), CTAS * L::kStageBytes);
+          const uint32_t fb = CTAS == 2 ? ptx::mapa(full_bar(s), 0) : full_bar(s);
+          auto load = [&](uint32_t dst, const CUtensorMap* map, int c0, int c1) {
+            if (CTAS == 2) ptx::tma_load_2d_pair(dst, map, fb, c0, c1); else ptx::tma_load_2d(dst, map, fb, c0, c1);
+          };
           const int k0 = kb * BK;
           if (A_MN) {
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j) ptx::tma_load_2d(a_dst + j * kAtomBytes, &tmA, full_bar(s), m0 + 64 * j, k0);
+            for (int j = 0; j < BM / 64; ++j) load(a_dst + j * kAtomBytes, &tmA, m0 + 64 * j, k0);
           } else {
-            ptx::tma_load_2d(a_dst, &tmA, full_bar(s), k0, m0);
+            load(a_dst, &tmA, k0, m0);
           }
           if (B_MN) {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j) ptx::tma_load_2d(b_dst + j * kAtomBytes, &tmB, full_bar(s), n0 + 64 * j, k0);
+            for (int j = 0; j < BN / CTAS / 64; ++j) load(b_dst + j * kAtomBytes, &tmB, n0 + 64 * j, k0);
           } else {
-            ptx::tma_load_2d(b_dst, &tmB, full_bar(s), k0, n0);
+            load(b_dst, &tmB, k0, n0);
           }
           ++issued;
           if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -240,12 +258,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, BN, A_MN, B_MN);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_bf16(BM * CTAS, BN, A_MN, B_MN);
+      auto commit = [&](uint32_t bar) {   // in a pair the barrier of both CTAs is signalled
+        if (CTAS == 2) ptx::mma_commit_pair(bar, 3); else ptx::mma_commit(bar);
+      };
       int s = 0; uint32_t ph = 0;
       int acc = 0; uint32_t aph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int tile = unit0; tile < num_tiles && ok; tile += unit_stride) {
         if (!ptx::mbar_wait_bounded(tempty_bar(acc), aph ^ 1u, abort_flag, kWaitLimitCycles)) {
           report_error(ep.status, STEM_ERR_TIMEOUT, 3);
           *abort_flag = 1; ok = false; break;
@@ -269,18 +290,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                      : ptx::make_smem_desc(a_src + kk * (UMMA_K * 2), 16, 1024);
             const uint64_t bd = B_MN ? ptx::make_smem_desc(b_src + kk * (UMMA_K * 128), kAtomBytes, 1024)
                                      : ptx::make_smem_desc(b_src + kk * (UMMA_K * 2), 16, 1024);
-            ptx::mma_bf16_ss(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
+            if (CTAS == 2) ptx::mma_bf16_ss_pair(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
+            else ptx::mma_bf16_ss(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
           }
-          ptx::mma_commit(empty_bar(s));
+          commit(empty_bar(s));
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
-        ptx::mma_commit(tfull_bar(acc));
+        commit(tfull_bar(acc));
         if (++acc == 2) { acc = 0; aph ^= 1u; }
       }
       if (!ok) {
         // let MMAs already issued finish before TMEM is freed
-        ptx::mma_commit(drain_bar);
+        if (CTAS == 2) ptx::mma_commit_pair(drain_bar, 1); else ptx::mma_commit(drain_bar);
         int zero = 0;
         ptx::mbar_wait_bounded(drain_bar, 0, &zero, kWaitLimitCycles);
       }
@@ -293,9 +315,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool second_out = KIND == kEpiDH || (KIND == kEpiGate && ep.G != nullptr);
     int acc = 0; uint32_t aph = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+    for (int tile = unit0; tile < num_tiles && ok; tile += unit_stride) {
       const TileCoord tc = tile_coord(tile, tiles_m, tiles_n, group_m);
-      const int m_warp = tc.m_blk * BM + q * 32;  // first row of this warp's 32-row block
+      const int m_warp = (tc.m_blk * CTAS + rank) * BM + q * 32;  // first row of this warp's 32-row block
       const int m = m_warp + lane;
       const int n0 = tc.n_blk * BN + half * (BN / 2);
       const bool row_ok = m < M;
@@ -342,7 +364,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           // the accumulator has been read out: hand it back to the MMA issuer
           ptx::tc_fence_before();
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+          if (lane == 0) {
+            if (rank == 0) ptx::mbar_arrive(tempty_bar(acc)); else ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(acc), 0));
+          }
         }
         // the staging buffer is free once the previous chunk's tensor stores have read it
         if (lane == 0) ptx::bulk_wait_read_all();
@@ -364,19 +388,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   __syncthreads();
   if (*abort_flag != 0 && threadIdx.x == 0) {
-    // wait (bounded) for TMA copies still in flight: the last issue into each stage
+    // wait (bounded) for TMA copies still in flight: the last issue into each stage.  The
+    // bytes of a pair's second CTA are counted on the first CTA's barriers, which it cannot
+    // poll; it waits out a fixed interval instead (far longer than a copy takes).
     int zero = 0;
-    for (int s = 0; s < STAGES; ++s) {
-      int last = -1;
-      for (int j = issued - 1; j >= 0 && j >= issued - STAGES; --j)
-        if (j % STAGES == s) { last = j; break; }
-      if (last >= 0) ptx::mbar_wait_bounded(full_bar(s), (last / STAGES) & 1, &zero, kWaitLimitCycles / 16);
+    if (rank == 0) {
+      for (int s = 0; s < STAGES; ++s) {
+        int last = -1;
+        for (int j = issued - 1; j >= 0 && j >= issued - STAGES; --j)
+          if (j % STAGES == s) { last = j; break; }
+        if (last >= 0) ptx::mbar_wait_bounded(full_bar(s), (last / STAGES) & 1, &zero, kWaitLimitCycles / 16);
+      }
+    } else {
+      const long long t0 = clock64();
+      while (clock64() - t0 < 2000000ll) { }
     }
   }
-  __syncthreads();
+  // Neither CTA of a pair may exit (or free TMEM) while the other can still signal its
+  // barriers, read its shared memory or write its accumulators.  Every role reaches this
+  // point in bounded time, so the cluster barrier cannot hang.
+  if (CTAS == 2) ptx::cluster_sync(); else __syncthreads();
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
+    if (CTAS == 2) ptx::tmem_dealloc_pair(tmem_base, kTmemCols); else ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -427,32 +461,47 @@ bool encode_out_map(CUtensorMap* map, const void* ptr, int rows, int cols, bool 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE>
+template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE, int CTAS>
 cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC0,
                         const CUtensorMap& tmC1, int M, int N, int K, const EpiParams& ep,
                         cudaStream_t stream) {
-  using L = Smem<BN, STAGES>;
-  auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES, WIDE>;
+  using L = Smem<BN, STAGES, CTAS>;
+  static_assert(L::kTotal <= 232448, "exceeds the shared memory a CTA can have");
+  auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES, WIDE, CTAS>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-  const int grid = tiles < device_sm_count() ? tiles : device_sm_count();
-    kern<<<grid, kThreads, L::kTotal, stream>>>(tmA, tmB, tmC0, tmC1, M, N, K, 8, ep);
+  // persistent: one CTA (or one pair) per SM (pair of SMs), each walking the tile list
+  const int units = ((M + BM * CTAS - 1) / (BM * CTAS)) * ((N + BN - 1) / BN);
+  const int slots = device_sm_count() / CTAS;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(CTAS * (units < slots ? units : slots)));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = L::kTotal;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC0, tmC1, M, N, K, 8, ep);
   count_launches(1);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-template <bool A_MN, bool B_MN, int KIND>
+template <bool A_MN, bool B_MN, int KIND, int CTAS>
 cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const EpiParams& ep,
                       cudaStream_t stream) {
-  constexpr int BN = 256, STAGES = 4;
+  // 192 KB of operand ring either way: 4 stages of 48 KB, or 6 stages of 32 KB per CTA of a pair
+  constexpr int BN = 256, STAGES = CTAS == 2 ? 6 : 4;
   CUtensorMap tmA, tmB;
   const bool okA = A_MN ? encode_map(&tmA, A, K, M, BK) : encode_map(&tmA, A, M, K, BM);
-  const bool okB = B_MN ? encode_map(&tmB, B, K, N, BK) : encode_map(&tmB, B, N, K, BN);
+  const bool okB = B_MN ? encode_map(&tmB, B, K, N, BK) : encode_map(&tmB, B, N, K, BN / CTAS);
   if (!okA || !okB) return cudaErrorNotSupported;
   CUtensorMap tmC0, tmC1;
   bool okC;
@@ -466,14 +515,21 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
   if (!okC) return cudaErrorNotSupported;
   auto a32 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; };
   const bool wide = (N % 16 == 0) && a32(ep.E) && a32(ep.Gin);
-  if (wide) return launch_inst<A_MN, B_MN, KIND, BN, STAGES, true>(tmA, tmB, tmC0, tmC1, M, N, K, ep, stream);
-  return launch_inst<A_MN, B_MN, KIND, BN, STAGES, false>(tmA, tmB, tmC0, tmC1, M, N, K, ep, stream);
+  if (wide) return launch_inst<A_MN, B_MN, KIND, BN, STAGES, true, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, stream);
+  return launch_inst<A_MN, B_MN, KIND, BN, STAGES, false, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, stream);
+}
+
+template <bool A_MN, bool B_MN, int KIND>
+cudaError_t launch_ctas(const void* A, const void* B, int M, int N, int K, const EpiParams& ep, bool pair,
+                        cudaStream_t stream) {
+  if (pair) return launch_bn<A_MN, B_MN, KIND, 2>(A, B, M, N, K, ep, stream);
+  return launch_bn<A_MN, B_MN, KIND, 1>(A, B, M, N, K, ep, stream);
 }
 
 }  // namespace
 
 cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const void* B, bool b_mn,
-                           EpiKind kind, const EpiParams& ep, cudaStream_t stream) {
+                           EpiKind kind, const EpiParams& ep, bool pair, cudaStream_t stream) {
   if (M <= 0 || N <= 0) return cudaSuccess;
   // TMA needs 16-byte row pitches (the contiguous extent of each operand a multiple of 8
   // elements); the epilogue stores 8 columns at a time.
@@ -481,15 +537,15 @@ cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const 
   // layer call sites: gate (K,K,gate)  down (K,K,store)  dH (K,MN,dh)  dx (K,MN,store)
   //                   dW_down / dW_gate (MN,MN,store); the plain-GEMM entry adds (MN,K,store)
   if (!a_mn && !b_mn) {
-    if (kind == kEpiGate) return launch_bn<false, false, kEpiGate>(A, B, M, N, K, ep, stream);
-    if (kind == kEpiStore) return launch_bn<false, false, kEpiStore>(A, B, M, N, K, ep, stream);
+    if (kind == kEpiGate) return launch_ctas<false, false, kEpiGate>(A, B, M, N, K, ep, pair, stream);
+    if (kind == kEpiStore) return launch_ctas<false, false, kEpiStore>(A, B, M, N, K, ep, pair, stream);
   } else if (!a_mn && b_mn) {
-    if (kind == kEpiDH) return launch_bn<false, true, kEpiDH>(A, B, M, N, K, ep, stream);
-    if (kind == kEpiStore) return launch_bn<false, true, kEpiStore>(A, B, M, N, K, ep, stream);
+    if (kind == kEpiDH) return launch_ctas<false, true, kEpiDH>(A, B, M, N, K, ep, pair, stream);
+    if (kind == kEpiStore) return launch_ctas<false, true, kEpiStore>(A, B, M, N, K, ep, pair, stream);
   } else if (a_mn && b_mn) {
-    if (kind == kEpiStore) return launch_bn<true, true, kEpiStore>(A, B, M, N, K, ep, stream);
+    if (kind == kEpiStore) return launch_ctas<true, true, kEpiStore>(A, B, M, N, K, ep, pair, stream);
   } else {
-    if (kind == kEpiStore) return launch_bn<true, false, kEpiStore>(A, B, M, N, K, ep, stream);
+    if (kind == kEpiStore) return launch_ctas<true, false, kEpiStore>(A, B, M, N, K, ep, pair, stream);
   }
   return cudaErrorNotSupported;
 }

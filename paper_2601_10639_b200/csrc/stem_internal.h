@@ -62,8 +62,9 @@ cudaError_t launch_simt_gemm(int dtype, int M, int N, int K, const void* A, bool
 
 // tcgen05 / TMEM / TMA kernels, bf16 inputs.  Returns cudaErrorNotSupported when the
 // shape cannot be described to TMA (the caller decides what to do).
+// pair: run on CTA pairs (cta_group::2, 256-row tiles) rather than single CTAs.
 cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const void* B,
-                           bool b_mn, EpiKind kind, const EpiParams& ep, cudaStream_t stream);
+                           bool b_mn, EpiKind kind, const EpiParams& ep, bool pair, cudaStream_t stream);
 
 // ---- index path ----------------------------------------------------------------------
 size_t dedup_workspace_bytes(int T, int V);

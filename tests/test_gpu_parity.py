@@ -26,7 +26,7 @@ def _ws():
 # ---------------------------------------------------------------------------------------
 # plain contraction, every operand layout, ragged tiles
 # ---------------------------------------------------------------------------------------
-@pytest.mark.parametrize("flags", [0, B.FLAG_SIMT], ids=["tcgen05", "fma"])
+@pytest.mark.parametrize("flags", [0, B.FLAG_SINGLE_CTA, B.FLAG_SIMT], ids=["tcgen05_pair", "tcgen05_single", "fma"])
 @pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 1), (1, 0)])
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (200, 328, 136), (512, 768, 1024), (8, 8, 8), (1000, 264, 520)])
 def test_gemm_layouts(flags, a_mn, b_mn, M, N, K):
@@ -128,7 +128,7 @@ def test_layer_fp32_config():
     _full_parity(w, synth.make_inputs(w), B.DTYPE_FP32, TOL_FP32)
 
 
-@pytest.mark.parametrize("flags", [0, B.FLAG_SIMT], ids=["tcgen05", "fma"])
+@pytest.mark.parametrize("flags", [0, B.FLAG_SINGLE_CTA, B.FLAG_SIMT], ids=["tcgen05_pair", "tcgen05_single", "fma"])
 @pytest.mark.parametrize("T,d,F,V,dist", [(300, 264, 520, 1000, "zipf"), (1024, 512, 768, 4096, "uniform"),
                                           (130, 64, 72, 50, "same"), (257, 1024, 2816, 32000, "zipf")])
 def test_layer_bf16_small(flags, T, d, F, V, dist):
