@@ -98,7 +98,7 @@ int check_shape(const stem_shape_t* s) {
 struct WsLayout {
   size_t dedup_off, dedup_bytes;
   size_t h_off, h_bytes;     // forward: H when the caller keeps none
-  size_t du_off, dg_off, tf_bytes, part_off, part_bytes;
+  size_t du_off, dg_off, tf_bytes, part_off, part_bytes, sk_off, sk_bytes;
   size_t total;
 };
 
@@ -114,9 +114,12 @@ WsLayout ws_layout(const stem_shape_t* s) {
   w.dg_off = w.du_off + tf;
   w.part_off = w.dg_off + tf;
   w.part_bytes = segreduce_workspace_bytes(s->T, s->d_ff);
+  // partial tiles of the token-contracted gradients (dW_down, dW_gate): live while dG is
+  w.sk_off = align_up(w.part_off + w.part_bytes, 1024);
+  w.sk_bytes = s->dtype == STEM_DTYPE_BF16 ? tc_gemm_scratch_bytes() : 0;
   size_t m = w.dedup_off + w.dedup_bytes;
   if (w.h_off + w.h_bytes > m) m = w.h_off + w.h_bytes;
-  if (w.part_off + w.part_bytes > m) m = w.part_off + w.part_bytes;
+  if (w.sk_off + w.sk_bytes > m) m = w.sk_off + w.sk_bytes;
   w.total = align_up(m, 256);
   return w;
 }
@@ -274,6 +277,7 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
   if (e != cudaSuccess) return cuda_fail(e);
   if (dW_down) {  // dW_down[i,j] = sum_t dy[t,i] H[t,j]
     EpiParams p; p.out = dW_down; p.out_fp32 = grad_fp32; p.status = status_of(ws);
+    p.sk_scratch = base + w.sk_off; p.sk_bytes = w.sk_bytes;
     ProfScope prof("dw_down_gemm", st);
     e = gemm(shape, d, F, T, dy, true, H_save, true, kEpiStore, p, st);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -286,6 +290,7 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
   }
   if (dW_gate) {  // dW_gate[j,k] = sum_t dG[t,j] x[t,k]
     EpiParams p; p.out = dW_gate; p.out_fp32 = grad_fp32; p.status = status_of(ws);
+    p.sk_scratch = base + w.sk_off; p.sk_bytes = w.sk_bytes;
     ProfScope prof("dw_gate_gemm", st);
     e = gemm(shape, F, d, T, dG, true, x, true, kEpiStore, p, st);
     if (e != cudaSuccess) return cuda_fail(e);

@@ -162,11 +162,37 @@ __device__ __forceinline__ TileCoord tile_coord(int tile, int tiles_m, int tiles
   return {first_m + in % gsize, in / gsize};
 }
 
+// ---- work list ----------------------------------------------------------------------------
+// Tiles [0, dp_tiles) are handed out whole, round robin over the P persistent CTAs (pairs).
+// When the tile count leaves a ragged last round, each of the remaining tiles is cut into
+// `split` pieces along k (equal k ranges) and the pieces are handed out round robin, ordered
+// k range first, so the pieces in flight together cover the same k range of different
+// tiles and share their operand panels in L2 exactly as whole tiles do.  A piece writes raw
+// fp32 sums to its slot of a partial-tile matrix; a small fix-up kernel adds each tile's
+// pieces in ascending k order, so the result does not depend on timing.
+struct Work { int tile, kb0, kb1, slot; };  // slot < 0: a whole tile, written to the output
+
+struct WorkList {
+  int p, P, dp_tiles, num_tiles, k_blocks, split;
+  // i-th work item of CTA (pair) p; false when the list is exhausted
+  __device__ __forceinline__ bool get(int i, Work& w) const {
+    const int n_dp = dp_tiles > p ? (dp_tiles - p + P - 1) / P : 0;
+    if (i < n_dp) { w = {p + i * P, 0, k_blocks, -1}; return true; }
+    const int tail = num_tiles - dp_tiles;
+    const int q = p + (i - n_dp) * P;          // piece number
+    if (q >= tail * split) return false;
+    const int ik = q / tail, j = q - ik * tail;  // k range, tail tile
+    w = {dp_tiles + j, static_cast<int>(static_cast<long long>(k_blocks) * ik / split),
+         static_cast<int>(static_cast<long long>(k_blocks) * (ik + 1) / split), q};
+    return true;
+  }
+};
+
 template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
-               int M, int N, int K, int group_m, EpiParams ep) {
+               int M, int N, int K, int group_m, int dp_tiles, int split, EpiParams ep) {
   using L = Smem<BN, STAGES, CTAS>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -189,6 +215,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int num_tiles = tiles_m * tiles_n;
   const int k_blocks = (K + BK - 1) / BK;
   constexpr uint32_t kTmemCols = 2 * BN;
+  const WorkList work{unit0, unit_stride, dp_tiles, num_tiles, k_blocks, split};
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
@@ -222,11 +249,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) {
       int s = 0; uint32_t ph = 0;
       bool ok = true;
-      for (int tile = unit0; tile < num_tiles && ok; tile += unit_stride) {
-        const TileCoord tc = tile_coord(tile, tiles_m, tiles_n, group_m);
+      Work w;
+      for (int i = 0; ok && work.get(i, w); ++i) {
+        const TileCoord tc = tile_coord(w.tile, tiles_m, tiles_n, group_m);
         // this CTA's rows of A and its share of the columns of B
         const int m0 = (tc.m_blk * CTAS + rank) * BM, n0 = tc.n_blk * BN + rank * (BN / CTAS);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, kWaitLimitCycles)) {
             report_error(ep.status, STEM_ERR_TIMEOUT, 1);
             *abort_flag = 1; ok = false; break;
@@ -266,14 +294,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int s = 0; uint32_t ph = 0;
       int acc = 0; uint32_t aph = 0;
       bool ok = true;
-      for (int tile = unit0; tile < num_tiles && ok; tile += unit_stride) {
+      Work w;
+      for (int i = 0; ok && work.get(i, w); ++i) {
         if (!ptx::mbar_wait_bounded(tempty_bar(acc), aph ^ 1u, abort_flag, kWaitLimitCycles)) {
           report_error(ep.status, STEM_ERR_TIMEOUT, 3);
           *abort_flag = 1; ok = false; break;
         }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitCycles)) {
             report_error(ep.status, STEM_ERR_TIMEOUT, 2);
             *abort_flag = 1; ok = false; break;
@@ -290,8 +319,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                      : ptx::make_smem_desc(a_src + kk * (UMMA_K * 2), 16, 1024);
             const uint64_t bd = B_MN ? ptx::make_smem_desc(b_src + kk * (UMMA_K * 128), kAtomBytes, 1024)
                                      : ptx::make_smem_desc(b_src + kk * (UMMA_K * 2), 16, 1024);
-            if (CTAS == 2) ptx::mma_bf16_ss_pair(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
-            else ptx::mma_bf16_ss(d_tmem, ad, bd, idesc, (kb | kk) != 0 ? 1u : 0u);
+            if (CTAS == 2) ptx::mma_bf16_ss_pair(d_tmem, ad, bd, idesc, (kb > w.kb0 || kk > 0) ? 1u : 0u);
+            else ptx::mma_bf16_ss(d_tmem, ad, bd, idesc, (kb > w.kb0 || kk > 0) ? 1u : 0u);
           }
           commit(empty_bar(s));
           if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -315,8 +344,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool second_out = KIND == kEpiDH || (KIND == kEpiGate && ep.G != nullptr);
     int acc = 0; uint32_t aph = 0;
     bool ok = true;
-    for (int tile = unit0; tile < num_tiles && ok; tile += unit_stride) {
-      const TileCoord tc = tile_coord(tile, tiles_m, tiles_n, group_m);
+    Work w;
+    for (int i = 0; ok && work.get(i, w); ++i) {
+      const TileCoord tc = tile_coord(w.tile, tiles_m, tiles_n, group_m);
       const int m_warp = (tc.m_blk * CTAS + rank) * BM + q * 32;  // first row of this warp's 32-row block
       const int m = m_warp + lane;
       const int n0 = tc.n_blk * BN + half * (BN / 2);
@@ -371,13 +401,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // the staging buffer is free once the previous chunk's tensor stores have read it
         if (lane == 0) ptx::bulk_wait_read_all();
         __syncwarp();
-        epilogue_row32<KIND>(ep, out_buf, lane, v, e_cur, g_cur);
-        ptx::fence_proxy_async();
-        __syncwarp();
-        if (lane == 0 && m_warp < M && n < N) {
-          ptx::tma_store_2d(&tmC0, out_buf, n, m_warp);
-          if (second_out) ptx::tma_store_2d(&tmC1, out_buf + 2048, n, m_warp);
-          ptx::bulk_commit_group();
+        if (KIND == kEpiStore && w.slot >= 0) {
+          // a piece of a tile: raw fp32 sums into the piece's slot of the partial-tile matrix
+          // (tmC1: [slots * BM * CTAS, BN] fp32), finished by the fix-up kernel
+          stage_row_f32(out_buf, lane, v);
+          ptx::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            ptx::tma_store_2d(&tmC1, out_buf, half * (BN / 2) + c * 32, (w.slot * CTAS + rank) * BM + q * 32);
+            ptx::bulk_commit_group();
+          }
+        } else {
+          epilogue_row32<KIND>(ep, out_buf, lane, v, e_cur, g_cur);
+          ptx::fence_proxy_async();
+          __syncwarp();
+          if (lane == 0 && m_warp < M && n < N) {
+            ptx::tma_store_2d(&tmC0, out_buf, n, m_warp);
+            if (second_out) ptx::tma_store_2d(&tmC1, out_buf + 2048, n, m_warp);
+            ptx::bulk_commit_group();
+          }
         }
       }
       if (++acc == 2) { acc = 0; aph ^= 1u; }
@@ -411,6 +453,38 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 1) {
     ptx::tc_fence_after();
     if (CTAS == 2) ptx::tmem_dealloc_pair(tmem_base, kTmemCols); else ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Fix-up for the tail tiles: output tile = sum of its pieces in ascending k order (piece ik of
+// tail tile j is slot ik * tail + j).  One CTA per (tail tile, 32-row band).
+template <int BN, int CTAS>
+__global__ void __launch_bounds__(256)
+tail_fixup_kernel(int M, int N, int dp_tiles, int tail, int split, int tiles_m, int tiles_n, int group_m,
+                  const float* __restrict__ partial, void* __restrict__ out, int out_fp32) {
+  constexpr int TM = BM * CTAS;
+  const int j = blockIdx.x;
+  const TileCoord tc = tile_coord(dp_tiles + j, tiles_m, tiles_n, group_m);
+  const int r0 = blockIdx.y * 32;
+  for (int e = threadIdx.x; e < 32 * (BN / 4); e += 256) {
+    const int r = r0 + e / (BN / 4), c = (e % (BN / 4)) * 4;
+    const int m = tc.m_blk * TM + r, nn = tc.n_blk * BN + c;
+    if (m >= M || nn >= N) continue;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int ik = 0; ik < split; ++ik) {
+      const size_t slot = static_cast<size_t>(ik) * tail + j;
+      const float4 v = *reinterpret_cast<const float4*>(partial + (slot * TM + r) * BN + c);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    const size_t o = static_cast<size_t>(m) * N + nn;   // N is a multiple of 8: 4 columns never straddle the edge
+    if (out_fp32) {
+      *reinterpret_cast<float4*>(static_cast<float*>(out) + o) = acc;
+    } else {
+      uint2 pk;
+      pk.x = pack_bf16(acc.x, acc.y);
+      pk.y = pack_bf16(acc.z, acc.w);
+      *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + o) = pk;
+    }
   }
 }
 
@@ -463,8 +537,8 @@ bool encode_out_map(CUtensorMap* map, const void* ptr, int rows, int cols, bool 
 
 template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE, int CTAS>
 cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC0,
-                        const CUtensorMap& tmC1, int M, int N, int K, const EpiParams& ep,
-                        cudaStream_t stream) {
+                        const CUtensorMap& tmC1, int M, int N, int K, const EpiParams& ep, int sk_tail,
+                        int sk_split, cudaStream_t stream) {
   using L = Smem<BN, STAGES, CTAS>;
   static_assert(L::kTotal <= 232448, "exceeds the shared memory a CTA can have");
   auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES, WIDE, CTAS>;
@@ -474,11 +548,14 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  // persistent: one CTA (or one pair) per SM (pair of SMs), each walking the tile list
-  const int units = ((M + BM * CTAS - 1) / (BM * CTAS)) * ((N + BN - 1) / BN);
+  // persistent: one CTA (or one pair) per SM (pair of SMs), each walking its work list
+  const int tiles_m = (M + BM * CTAS - 1) / (BM * CTAS), tiles_n = (N + BN - 1) / BN;
+  const int units = tiles_m * tiles_n;
   const int slots = device_sm_count() / CTAS;
+  const int P = sk_tail > 0 ? slots : (units < slots ? units : slots);
+  const int dp_tiles = sk_tail > 0 ? units - sk_tail : units;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(CTAS * (units < slots ? units : slots)));
+  cfg.gridDim = dim3(static_cast<unsigned>(CTAS * P));
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = L::kTotal;
   cfg.stream = stream;
@@ -489,8 +566,14 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC0, tmC1, M, N, K, 8, ep);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC0, tmC1, M, N, K, 8, dp_tiles, sk_split, ep);
   count_launches(1);
+  if (e == cudaSuccess && sk_tail > 0) {
+    tail_fixup_kernel<BN, CTAS><<<dim3(sk_tail, BM * CTAS / 32), 256, 0, stream>>>(
+        M, N, dp_tiles, sk_tail, sk_split, tiles_m, tiles_n, 8, static_cast<const float*>(ep.sk_scratch), ep.out,
+        ep.out_fp32);
+    count_launches(1);
+  }
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -505,9 +588,34 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
   if (!okA || !okB) return cudaErrorNotSupported;
   CUtensorMap tmC0, tmC1;
   bool okC;
+  int sk_tail = 0, sk_split = 1;  // tiles of the ragged last round, pieces per tile along k
   if (KIND == kEpiStore) {
     okC = encode_out_map(&tmC0, ep.out, M, N, ep.out_fp32 != 0);
     tmC1 = tmC0;
+    // The last round costs ceil(tail * split / slots) / split tile times instead of one.
+    // Worth it when that saves clearly more than the partial tiles and the fix-up launch
+    // cost (~25 us); a tile time is ~ 2 TM BN K flops at ~11 TFLOP/s per SM.
+    constexpr int TM = BM * CTAS;
+    const int units = ((M + TM - 1) / TM) * ((N + BN - 1) / BN);
+    const int slots = device_sm_count() / CTAS;
+    const int k_blocks = (K + BK - 1) / BK;
+    const int tail = units % slots;
+    const size_t slot_bytes = static_cast<size_t>(TM) * BN * sizeof(float);
+    const double tile_us = 2.0 * TM * BN * static_cast<double>(K) / (11.0e6 * CTAS);
+    if (tail > 0 && ep.sk_scratch != nullptr) {
+      int best = 1;
+      double best_cost = 1.0;
+      for (int sp = 2; sp <= 8; ++sp) {
+        if (static_cast<size_t>(tail) * sp * slot_bytes > ep.sk_bytes || k_blocks / sp < 4) break;
+        const double cost = static_cast<double>((tail * sp + slots - 1) / slots) / sp;
+        if (cost < best_cost - 0.04) { best_cost = cost; best = sp; }
+      }
+      if (best > 1 && (1.0 - best_cost) * tile_us > 25.0) {
+        sk_tail = tail;
+        sk_split = best;
+        okC = okC && encode_out_map(&tmC1, ep.sk_scratch, tail * best * TM, BN, true);
+      }
+    }
   } else {
     okC = encode_out_map(&tmC0, ep.H, M, N, false);
     if (ep.G) okC = okC && encode_out_map(&tmC1, ep.G, M, N, false); else tmC1 = tmC0;
@@ -515,8 +623,8 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
   if (!okC) return cudaErrorNotSupported;
   auto a32 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; };
   const bool wide = (N % 16 == 0) && a32(ep.E) && a32(ep.Gin);
-  if (wide) return launch_inst<A_MN, B_MN, KIND, BN, STAGES, true, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, stream);
-  return launch_inst<A_MN, B_MN, KIND, BN, STAGES, false, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, stream);
+  if (wide) return launch_inst<A_MN, B_MN, KIND, BN, STAGES, true, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, sk_tail, sk_split, stream);
+  return launch_inst<A_MN, B_MN, KIND, BN, STAGES, false, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, sk_tail, sk_split, stream);
 }
 
 template <bool A_MN, bool B_MN, int KIND>
@@ -527,6 +635,12 @@ cudaError_t launch_ctas(const void* A, const void* B, int M, int N, int K, const
 }
 
 }  // namespace
+
+size_t tc_gemm_scratch_bytes() {
+  // room for 296 partial 256 x 256 fp32 tiles: up to four pieces for each of the at most 73
+  // tail tiles of a pair launch (twice as many 128 x 256 tiles for single CTAs)
+  return static_cast<size_t>(4) * 148 * 128 * 256 * sizeof(float);
+}
 
 cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const void* B, bool b_mn,
                            EpiKind kind, const EpiParams& ep, bool pair, cudaStream_t stream) {

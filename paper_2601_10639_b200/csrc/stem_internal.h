@@ -52,6 +52,10 @@ struct EpiParams {
   void* G = nullptr;    // kEpiGate: G out (opt.)   kEpiDH: dG out
   const void* Gin = nullptr;  // kEpiDH: saved G
   int32_t* status = nullptr;
+  // kEpiStore, optional: scratch for partial tiles when the last round of tiles is split
+  // along k (tc_gemm_scratch_bytes()); without it every tile is computed whole
+  void* sk_scratch = nullptr;
+  size_t sk_bytes = 0;
 };
 
 // C[m,n] = sum_k A(m,k) B(n,k); a_mn/b_mn: operand stored with the M (N) index contiguous.
@@ -65,6 +69,8 @@ cudaError_t launch_simt_gemm(int dtype, int M, int N, int K, const void* A, bool
 // pair: run on CTA pairs (cta_group::2, 256-row tiles) rather than single CTAs.
 cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const void* B,
                            bool b_mn, EpiKind kind, const EpiParams& ep, bool pair, cudaStream_t stream);
+
+size_t tc_gemm_scratch_bytes();
 
 // ---- index path ----------------------------------------------------------------------
 size_t dedup_workspace_bytes(int T, int V);

@@ -136,6 +136,15 @@ def test_layer_bf16_small(flags, T, d, F, V, dist):
     _full_parity(w, synth.make_inputs(w, seed=77), B.DTYPE_BF16, TOL_BF16, flags)
 
 
+@pytest.mark.parametrize("flags", [0, B.FLAG_SINGLE_CTA], ids=["pair", "single"])
+@pytest.mark.parametrize("T,d,F,grad", [(8192, 256, 512, B.DTYPE_FP32), (8200, 264, 520, B.DTYPE_BF16)])
+def test_layer_bf16_many_tokens_few_tiles(flags, T, d, F, grad):
+    """Token-contracted gradients with fewer output tiles than SMs: the k range of each tile is
+    split over CTAs and summed by the fix-up kernel."""
+    w = synth.Workload("t", T, d, F, 2000, "bf16", "zipf")
+    _full_parity(w, synth.make_inputs(w, seed=90), B.DTYPE_BF16, TOL_BF16, flags, grad_dtype=grad)
+
+
 def test_layer_bf16_grad_bf16():
     w = synth.Workload("t", 512, 256, 512, 300, "bf16", "zipf")
     _full_parity(w, synth.make_inputs(w, seed=78), B.DTYPE_BF16, TOL_BF16, 0, grad_dtype=B.DTYPE_BF16)
