@@ -5,10 +5,9 @@
 // per (block, column slab) walks its positions in order, accumulating in fp32 registers.
 // A run whose segment lies wholly inside the block is final and is written to dE_rows; a
 // run whose segment crosses a block edge (at most the first and the last run of a block)
-// goes to a partial row, and the block in which such a segment starts is appended to a
-// list.  Pass 2: one CTA per list entry adds that segment's partial rows.  The order of the
-// list varies from run to run (an integer atomic hands out its slots) but each entry is
-// handled on its own and every summation order depends on the index arrays only, so the
+// goes to a partial row, and every block records which segment (if any) starts inside it and
+// runs past its end.  Pass 2: the CTAs of such a block add that segment's partial rows; the
+// others exit at once.  Every summation order depends on the index arrays only, so the
 // result is bitwise reproducible.  HBM-bound: every dU row is read once with 16-byte loads,
 // coalesced along d_ff.
 #include "stem_internal.h"
@@ -63,17 +62,17 @@ __device__ __forceinline__ void store_row(TOut* dst, const float (&v)[VI]) {
   for (int i = 0; i < VI; i += Vec<TOut>::N) Vec<TOut>::store(dst + i, v + i);
 }
 
-// Scratch layout: [0] number of entries in the list of crossing segments, [1..n_blk] the
-// list (block in which each crossing segment starts), then 2 partial rows per block.
+// Scratch layout: cross_seg[n_blk] (segment that starts in the block and crosses its end, or
+// -1), then 2 partial rows per block.
 __host__ __device__ inline size_t partial_offset_bytes(int n_blk) {
-  return (static_cast<size_t>(n_blk + 1) * 4 + 255) / 256 * 256;
+  return (static_cast<size_t>(n_blk) * 4 + 255) / 256 * 256;
 }
 
 template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(kThreads, 6)
 segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* __restrict__ perm,
                        const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ n_unique,
-                       TOut* __restrict__ dE_rows, int32_t* __restrict__ cross_list,
+                       TOut* __restrict__ dE_rows, int32_t* __restrict__ cross_seg,
                        float* __restrict__ partial) {
   constexpr int VI = (Vec<TIn>::N > Vec<TOut>::N) ? Vec<TIn>::N : Vec<TOut>::N;
   constexpr int LD = VI / Vec<TIn>::N;  // 16-byte loads per row per thread
@@ -118,7 +117,7 @@ segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* 
   if (blockIdx.y == 0 && threadIdx.x == 0) {
     // a segment that starts in this block and runs past its end is finished by pass 2
     const int j = s_loc[cnt - 1];
-    if (s_off[j] >= p0 && s_off[j + 1] > p0 + kSegBlk) cross_list[1 + atomicAdd(cross_list, 1)] = blk;
+    cross_seg[blk] = (s_off[j] >= p0 && s_off[j + 1] > p0 + kSegBlk) ? r_first + j : -1;
   }
   const int col = (blockIdx.y * kThreads + threadIdx.x) * VI;
   if (col >= F) return;
@@ -161,63 +160,48 @@ segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* 
   }
 }
 
-// One CTA per (crossing segment, 32 x VI columns): kRowLanes partial rows are added side by
-// side, each lane walking its rows in block order, then the lanes are combined in lane order.
+// One CTA per (block, 32 x VI columns); only blocks in which a crossing segment starts do
+// work: kRowLanes partial rows are added side by side, each lane walking its rows in block
+// order, then the lanes are combined in lane order.
 template <typename TOut, int VI>
 __global__ void __launch_bounds__(kRowLanes * kColLanes, 4)
 segreduce_pass2_kernel(int T, int F, const int32_t* __restrict__ seg_offsets,
-                       const int32_t* __restrict__ n_unique, const int32_t* __restrict__ cross_list,
-                       const float* __restrict__ partial, TOut* __restrict__ dE_rows) {
+                       const int32_t* __restrict__ cross_seg, const float* __restrict__ partial,
+                       TOut* __restrict__ dE_rows) {
   __shared__ float s_sum[kRowLanes][kColLanes][VI + 1];
-  __shared__ int s_r;
-  const int n_cross = cross_list[0];
-  const int n_u = *n_unique;
+  const int blk = blockIdx.x;
+  const int r = cross_seg[blk];
+  if (r < 0) return;
   const int cl = threadIdx.x % kColLanes, rl = threadIdx.x / kColLanes;
   const int col = (blockIdx.y * kColLanes + cl) * VI;
-  for (int e = blockIdx.x; e < n_cross; e += gridDim.x) {
-    const int blk = cross_list[1 + e];
-    const int p0 = blk * kSegBlk;
-    if (threadIdx.x == 0) {
-      // the segment of the block's last position
-      const int p_last = min(T, p0 + kSegBlk) - 1;
-      int lo = 0, hi = n_u;
-      while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (seg_offsets[mid] <= p_last) lo = mid; else hi = mid;
-      }
-      s_r = lo;
-    }
-    __syncthreads();
-    const int r = s_r;
-    const int seg_begin = seg_offsets[r], seg_end = seg_offsets[r + 1];
-    const int b_last = (seg_end - 1) / kSegBlk;
-    float acc[VI];
+  const int p0 = blk * kSegBlk;
+  const int seg_begin = seg_offsets[r], seg_end = seg_offsets[r + 1];
+  const int b_last = (seg_end - 1) / kSegBlk;
+  float acc[VI];
 #pragma unroll
-    for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
-    if (col < F) {
-      for (int b = blk + rl; b <= b_last; b += kRowLanes) {
-        // the segment's run is the first run of block b, unless b is the block it starts in
-        // and it does not start at that block's first position
-        const int slot = (b > blk || seg_begin == p0) ? 2 * b : 2 * b + 1;
-        const float* src = partial + static_cast<size_t>(slot) * F + col;
+  for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
+  if (col < F) {
+    for (int b = blk + rl; b <= b_last; b += kRowLanes) {
+      // the segment's run is the first run of block b, unless b is the block it starts in
+      // and it does not start at that block's first position
+      const int slot = (b > blk || seg_begin == p0) ? 2 * b : 2 * b + 1;
+      const float* src = partial + static_cast<size_t>(slot) * F + col;
 #pragma unroll
-        for (int i = 0; i < VI; i += 4) {
-          const float4 q = *reinterpret_cast<const float4*>(src + i);
-          acc[i] += q.x; acc[i + 1] += q.y; acc[i + 2] += q.z; acc[i + 3] += q.w;
-        }
+      for (int i = 0; i < VI; i += 4) {
+        const float4 q = *reinterpret_cast<const float4*>(src + i);
+        acc[i] += q.x; acc[i + 1] += q.y; acc[i + 2] += q.z; acc[i + 3] += q.w;
       }
     }
+  }
 #pragma unroll
-    for (int i = 0; i < VI; ++i) s_sum[rl][cl][i] = acc[i];
-    __syncthreads();
-    if (rl == 0 && col < F) {
+  for (int i = 0; i < VI; ++i) s_sum[rl][cl][i] = acc[i];
+  __syncthreads();
+  if (rl == 0 && col < F) {
 #pragma unroll
-      for (int l = 1; l < kRowLanes; ++l)
+    for (int l = 1; l < kRowLanes; ++l)
 #pragma unroll
-        for (int i = 0; i < VI; ++i) acc[i] += s_sum[l][cl][i];
-      store_row<VI, TOut>(dE_rows + static_cast<size_t>(r) * F + col, acc);
-    }
-    __syncthreads();
+      for (int i = 0; i < VI; ++i) acc[i] += s_sum[l][cl][i];
+    store_row<VI, TOut>(dE_rows + static_cast<size_t>(r) * F + col, acc);
   }
 }
 
@@ -226,17 +210,15 @@ cudaError_t launch_typed(int T, int F, const void* dU, const int32_t* perm, cons
                          const int32_t* n_unique, void* dE_rows, void* scratch, cudaStream_t stream) {
   constexpr int VI = (Vec<TIn>::N > Vec<TOut>::N) ? Vec<TIn>::N : Vec<TOut>::N;
   const int n_blk = (T + kSegBlk - 1) / kSegBlk;
-  int32_t* cross_list = static_cast<int32_t*>(scratch);
+  int32_t* cross_seg = static_cast<int32_t*>(scratch);
   float* partial = reinterpret_cast<float*>(static_cast<char*>(scratch) + partial_offset_bytes(n_blk));
-  cudaError_t e = cudaMemsetAsync(cross_list, 0, sizeof(int32_t), stream);
-  if (e != cudaSuccess) return e;
   dim3 grid1(n_blk, (F + kThreads * VI - 1) / (kThreads * VI));
   segreduce_pass1_kernel<TIn, TOut><<<grid1, kThreads, 0, stream>>>(
-      T, F, static_cast<const TIn*>(dU), perm, seg_offsets, n_unique, static_cast<TOut*>(dE_rows), cross_list,
+      T, F, static_cast<const TIn*>(dU), perm, seg_offsets, n_unique, static_cast<TOut*>(dE_rows), cross_seg,
       partial);
-  dim3 grid2(n_blk < 64 ? n_blk : 64, (F + kColLanes * VI - 1) / (kColLanes * VI));
+  dim3 grid2(n_blk, (F + kColLanes * VI - 1) / (kColLanes * VI));
   segreduce_pass2_kernel<TOut, VI><<<grid2, kRowLanes * kColLanes, 0, stream>>>(
-      T, F, seg_offsets, n_unique, cross_list, partial, static_cast<TOut*>(dE_rows));
+      T, F, seg_offsets, cross_seg, partial, static_cast<TOut*>(dE_rows));
   count_launches(2);
   return cudaGetLastError();
 }
