@@ -208,9 +208,18 @@ int stem_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t a_mn,
  * host_*: host memory ([T,d_model] in dtype; ids [T] int32), page-locked for the copies
  * to be asynchronous.  W_gate, E, W_down: device-resident parameters.  dW_gate, dW_down,
  * dE_rows, unique_ids [min(T,V)], n_unique [1]: device outputs, as in stem_ffn_backward
- * (they stay on the device for the optimizer).  arena: device scratch of
- * stem_step_arena_bytes() bytes holding the workspace (call stem_init_workspace on it
- * once) and every intermediate.  Everything is enqueued on `stream`.
+ * (they stay on the device for the optimizer; valid in `stream` order).  arena: device
+ * scratch of stem_step_arena_bytes() bytes holding the workspace (call stem_init_workspace
+ * on it once), every intermediate, and two slots of input and output buffers.
+ * Pipelining: the kernels run on `stream`; the copies run on two copy streams the library
+ * creates per device on first use (host-side objects only), chained to the kernels with
+ * events.  Successive calls alternate between the two slots, so the host-to-device copy
+ * of call k+1 and the device-to-host copy of call k-1 overlap the kernels of call k.
+ * Consequences for the caller: the host INPUT buffers of a call must stay unchanged, and
+ * its host OUTPUT buffers are not complete, until stem_ffn_step_host_flush(stream) has
+ * been called and `stream` synchronised (flush makes `stream` wait for every outstanding
+ * output copy; it is cheap and may be called after every step at the price of the
+ * overlap).  Calls on one device are serialised by a lock; use one arena at a time.
  */
 int stem_step_arena_bytes(const stem_shape_t* shape, size_t* bytes /*host, out*/);
 int stem_ffn_step_host(const stem_shape_t* shape, const void* host_x, const int32_t* host_ids,
@@ -218,6 +227,7 @@ int stem_ffn_step_host(const stem_shape_t* shape, const void* host_x, const int3
                        void* host_y, void* host_dx, void* dW_gate, void* dW_down, void* dE_rows,
                        int32_t* unique_ids, int32_t* n_unique, int32_t* host_n_unique /*host*/,
                        void* arena, size_t arena_bytes, void* stream);
+int stem_ffn_step_host_flush(void* stream);
 
 /*
  * Instrumentation (no counterpart in the paper).  stem_launch_count: kernels this library

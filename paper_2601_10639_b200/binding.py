@@ -29,7 +29,7 @@ EXPORTS = (
     "stem_version", "stem_status_string", "stem_workspace_bytes", "stem_init_workspace",
     "stem_query_status", "stem_dedup_ids", "stem_ffn_forward", "stem_ffn_backward",
     "stem_prefetch_rows", "stem_writeback_rows", "stem_gemm_bf16", "stem_step_arena_bytes",
-    "stem_ffn_step_host", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
+    "stem_ffn_step_host", "stem_ffn_step_host_flush", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
     "stem_dedup_ids_static", "stem_dedup_static_max_tokens",
 )
 
@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
             "stem_dedup_ids_static": [shp, vp, vp, vp, vp, vp, vp, vp, vp],
             "stem_dedup_static_max_tokens": [],
             "stem_ffn_step_host": [shp] + [vp] * 15 + [sz, vp],
+            "stem_ffn_step_host_flush": [vp],
             "stem_profile_enable": [ctypes.c_int],
             "stem_profile_count": [],
             "stem_profile_get": [ctypes.c_int, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float)],
@@ -186,6 +187,11 @@ def stem_ffn_step_host(shape, host_x, host_ids, host_dy, W_gate, E, W_down, host
                                     _p(W_down), _p(host_y), _p(host_dx), _p(dW_gate), _p(dW_down), _p(dE_rows),
                                     _p(unique_ids), _p(n_unique), _p(host_n_unique), _p(arena),
                                     arena.numel() * arena.element_size(), _stream(stream)), "stem_ffn_step_host")
+
+
+def stem_ffn_step_host_flush(stream=None) -> None:
+    """Make `stream` wait for the output copies of every stem_ffn_step_host call so far."""
+    _check(lib().stem_ffn_step_host_flush(_stream(stream)), "stem_ffn_step_host_flush")
 
 
 def stem_launch_count() -> int:

@@ -386,8 +386,11 @@ int stem_profile_get(int i, const char** name, float* ms) {
 }
 
 namespace {
+// Arena of the host-buffer step: the workspace, the saved activations and index arrays, and
+// TWO slots of input (x, dy, ids) and output (y, dx) buffers, so the copies of one call
+// overlap the kernels of its neighbours.
 struct Arena {
-  size_t ws, ws_bytes, x, dy, ids, y, dx, G, H, inverse, perm, seg, total;
+  size_t ws, ws_bytes, x[2], dy[2], ids[2], y[2], dx[2], G, H, inverse, perm, seg, total;
 };
 Arena arena_layout(const stem_shape_t* s) {
   Arena a{};
@@ -396,11 +399,44 @@ Arena arena_layout(const stem_shape_t* s) {
   const size_t R = static_cast<size_t>(s->T < s->V ? s->T : s->V);
   size_t o = 0;
   a.ws = o; a.ws_bytes = ws_layout(s).total; o += a.ws_bytes;
-  a.x = o; o += td;  a.dy = o; o += td;  a.ids = o; o += ti;
-  a.y = o; o += td;  a.dx = o; o += td;  a.G = o; o += tf;  a.H = o; o += tf;
+  for (int k = 0; k < 2; ++k) {
+    a.x[k] = o; o += td;  a.dy[k] = o; o += td;  a.ids[k] = o; o += ti;
+    a.y[k] = o; o += td;  a.dx[k] = o; o += td;
+  }
+  a.G = o; o += tf;  a.H = o; o += tf;
   a.inverse = o; o += ti;  a.perm = o; o += ti;  a.seg = o; o += align_up((R + 1) * 4, 256);
   a.total = o;
   return a;
+}
+
+// Copy streams and hand-over events of the host-buffer step, one set per device, created on
+// first use (host-side objects; no device memory).
+struct StepPipe {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t x_in[2], dy_in[2], y_done[2], bwd_done[2], out_done[2];
+  bool used[2] = {false, false};
+  unsigned long long calls = 0;
+};
+std::mutex g_pipe_mutex;
+StepPipe g_pipe[64];
+
+cudaError_t pipe_get(StepPipe** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  StepPipe& p = g_pipe[dev];
+  if (!p.ready) {
+    if ((e = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    if ((e = cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    for (int k = 0; k < 2; ++k)
+      for (cudaEvent_t* ev : {&p.x_in[k], &p.dy_in[k], &p.y_done[k], &p.bwd_done[k], &p.out_done[k]})
+        if ((e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming)) != cudaSuccess) return e;
+    p.ready = true;
+  }
+  *out = &p;
+  return cudaSuccess;
 }
 }  // namespace
 
@@ -422,34 +458,64 @@ int stem_ffn_step_host(const stem_shape_t* shape, const void* host_x, const int3
   const Arena a = arena_layout(shape);
   if (arena_bytes < a.total) return STEM_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  StepPipe* pp = nullptr;
+  cudaError_t e = pipe_get(&pp);
+  if (e != cudaSuccess) return cuda_fail(e);
+  StepPipe& p = *pp;
+  const int k = static_cast<int>(p.calls++ & 1);   // slot of this call
   char* base = static_cast<char*>(arena);
   const size_t td = static_cast<size_t>(shape->T) * shape->d_model * elem_bytes(shape->dtype);
-  cudaError_t e;
-  {
-    ProfScope prof("h2d_inputs", st);
-    e = cudaMemcpyAsync(base + a.ids, host_ids, static_cast<size_t>(shape->T) * 4, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(base + a.x, host_x, td, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(base + a.dy, host_dy, td, cudaMemcpyHostToDevice, st);
-  }
-  if (e != cudaSuccess) return cuda_fail(e);
-  int32_t* ids = reinterpret_cast<int32_t*>(base + a.ids);
+  int32_t* ids = reinterpret_cast<int32_t*>(base + a.ids[k]);
   int32_t* perm = reinterpret_cast<int32_t*>(base + a.perm);
   int32_t* seg = reinterpret_cast<int32_t*>(base + a.seg);
+#define STEP_CUDA(call) do { e = (call); if (e != cudaSuccess) return cuda_fail(e); } while (0)
+  // inputs: the slot is free once the backward pass of the call that used it last is done
+  if (p.used[k]) STEP_CUDA(cudaStreamWaitEvent(p.in, p.bwd_done[k], 0));
+  {
+    ProfScope prof("h2d_inputs", p.in);
+    STEP_CUDA(cudaMemcpyAsync(ids, host_ids, static_cast<size_t>(shape->T) * 4, cudaMemcpyHostToDevice, p.in));
+    STEP_CUDA(cudaMemcpyAsync(base + a.x[k], host_x, td, cudaMemcpyHostToDevice, p.in));
+    STEP_CUDA(cudaEventRecord(p.x_in[k], p.in));
+    STEP_CUDA(cudaMemcpyAsync(base + a.dy[k], host_dy, td, cudaMemcpyHostToDevice, p.in));
+    STEP_CUDA(cudaEventRecord(p.dy_in[k], p.in));
+  }
+  // compute on the caller's stream; y/dx of this slot must have left for the host first
+  STEP_CUDA(cudaStreamWaitEvent(st, p.x_in[k], 0));
+  if (p.used[k]) STEP_CUDA(cudaStreamWaitEvent(st, p.out_done[k], 0));
   if (int rc = stem_dedup_ids(shape, ids, unique_ids, n_unique, reinterpret_cast<int32_t*>(base + a.inverse), perm, seg,
                               base + a.ws, a.ws_bytes, stream)) return rc;
-  if (int rc = stem_ffn_forward(shape, base + a.x, ids, W_gate, E, W_down, base + a.y, base + a.G, base + a.H,
+  if (int rc = stem_ffn_forward(shape, base + a.x[k], ids, W_gate, E, W_down, base + a.y[k], base + a.G, base + a.H,
                                 base + a.ws, a.ws_bytes, stream)) return rc;
-  if (int rc = stem_ffn_backward(shape, base + a.dy, base + a.x, ids, W_gate, E, W_down, base + a.G, base + a.H, perm,
-                                 seg, n_unique, base + a.dx, dW_gate, dW_down, dE_rows, unique_ids, base + a.ws,
-                                 a.ws_bytes, stream)) return rc;
+  STEP_CUDA(cudaEventRecord(p.y_done[k], st));
+  STEP_CUDA(cudaStreamWaitEvent(st, p.dy_in[k], 0));
+  if (int rc = stem_ffn_backward(shape, base + a.dy[k], base + a.x[k], ids, W_gate, E, W_down, base + a.G, base + a.H,
+                                 perm, seg, n_unique, base + a.dx[k], dW_gate, dW_down, dE_rows, unique_ids,
+                                 base + a.ws, a.ws_bytes, stream)) return rc;
+  STEP_CUDA(cudaEventRecord(p.bwd_done[k], st));
+  // outputs
+  STEP_CUDA(cudaStreamWaitEvent(p.out, p.y_done[k], 0));
   {
-    ProfScope prof("d2h_outputs", st);
-    e = cudaMemcpyAsync(host_y, base + a.y, td, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(host_dx, base + a.dx, td, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess && host_n_unique)
-      e = cudaMemcpyAsync(host_n_unique, n_unique, 4, cudaMemcpyDeviceToHost, st);
+    ProfScope prof("d2h_outputs", p.out);
+    STEP_CUDA(cudaMemcpyAsync(host_y, base + a.y[k], td, cudaMemcpyDeviceToHost, p.out));
+    STEP_CUDA(cudaStreamWaitEvent(p.out, p.bwd_done[k], 0));
+    STEP_CUDA(cudaMemcpyAsync(host_dx, base + a.dx[k], td, cudaMemcpyDeviceToHost, p.out));
+    if (host_n_unique) STEP_CUDA(cudaMemcpyAsync(host_n_unique, n_unique, 4, cudaMemcpyDeviceToHost, p.out));
   }
-  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+  STEP_CUDA(cudaEventRecord(p.out_done[k], p.out));
+  p.used[k] = true;
+  return STEM_OK;
+}
+
+int stem_ffn_step_host_flush(void* stream) {
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  StepPipe* pp = nullptr;
+  cudaError_t e = pipe_get(&pp);
+  if (e != cudaSuccess) return cuda_fail(e);
+  for (int k = 0; k < 2; ++k)
+    if (pp->used[k]) STEP_CUDA(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), pp->out_done[k], 0));
+#undef STEP_CUDA
+  return STEM_OK;
 }
 
 }  // extern "C"

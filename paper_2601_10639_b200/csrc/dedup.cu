@@ -19,7 +19,7 @@ constexpr int kMaxCtas = 64;
 // histogram per CTA) small enough for every CTA to re-derive its offsets by itself.
 struct Split { int n_ctas, epw; };
 __host__ __device__ inline Split make_split(int T) {
-  int n_ctas = (T + 4095) / 4096;
+  int n_ctas = (T + 1023) / 1024;
   n_ctas = n_ctas < 1 ? 1 : (n_ctas > kMaxCtas ? kMaxCtas : n_ctas);
   const int per_cta = (T + n_ctas - 1) / n_ctas;
   const int epw = ((per_cta + kWarps - 1) / kWarps + 31) / 32 * 32;

@@ -277,6 +277,49 @@ def test_host_table_prefetch_and_writeback():
     assert np.array_equal(cache[:n_u].float().cpu().numpy(), expect)
 
 
+def test_step_from_host_buffers_pipelined():
+    """Three back-to-back calls with different batches (the two buffer slots are both reused):
+    each must return exactly what the device-resident path computes for its batch."""
+    w = synth.Workload("t", 700, 256, 520, 900, "bf16", "zipf")
+    shape = B.make_shape(w.T, w.d_model, w.d_ff, w.V, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    arena = torch.empty(B.stem_step_arena_bytes(shape), dtype=torch.uint8, device="cuda")
+    B.stem_init_workspace(arena)
+    calls = []
+    for seed in (91, 92, 93):
+        inp = synth.make_inputs(w, seed=seed)
+        st = runner.state_from_numpy(inp, B.DTYPE_BF16, w.V)
+        st.step()
+        torch.cuda.synchronize()
+        host = {k: getattr(st, k).cpu().pin_memory() for k in ("x", "dy", "ids")}
+        out = {"y": torch.zeros_like(host["x"]).pin_memory(), "dx": torch.zeros_like(host["x"]).pin_memory(),
+               "n": torch.zeros(1, dtype=torch.int32).pin_memory()}
+        dev = {k: torch.zeros_like(st.bufs[k]) for k in ("dW_gate", "dW_down", "dE_rows", "unique_ids", "n_unique")}
+        calls.append((st, host, out, dev))
+    st0 = calls[0][0]
+    for st, host, out, dev in calls:       # same weights for every call; only the batch changes
+        B.stem_ffn_step_host(shape, host["x"], host["ids"], host["dy"], st0.W_gate, st0.E, st0.W_down, out["y"],
+                             out["dx"], dev["dW_gate"], dev["dW_down"], dev["dE_rows"], dev["unique_ids"],
+                             dev["n_unique"], out["n"], arena)
+    B.stem_ffn_step_host_flush()
+    torch.cuda.synchronize()
+    assert B.stem_query_status(arena) == B.OK
+    for i, (st, host, out, dev) in enumerate(calls):
+        if i > 0:                          # reference for this batch with the first call's weights
+            st.W_gate, st.E, st.W_down = st0.W_gate, st0.E, st0.W_down
+            st.step()
+            torch.cuda.synchronize()
+        n_u = int(st.bufs["n_unique"].item())
+        assert int(out["n"][0]) == n_u, i
+        assert torch.equal(out["y"], st.bufs["y"].cpu()), i
+        assert torch.equal(out["dx"], st.bufs["dx"].cpu()), i
+    # the device-side gradients are those of the last call
+    st = calls[-1][0]
+    n_u = int(st.bufs["n_unique"].item())
+    dev = calls[-1][3]
+    assert torch.equal(dev["dW_gate"], st.bufs["dW_gate"]) and torch.equal(dev["dW_down"], st.bufs["dW_down"])
+    assert torch.equal(dev["dE_rows"][:n_u], st.bufs["dE_rows"][:n_u])
+
+
 def test_error_paths_on_device_box():
     w = synth.Workload("t", 64, 64, 64, 10, "bf16", "uniform")
     inp = synth.make_inputs(w, seed=81)
