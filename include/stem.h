@@ -187,6 +187,18 @@ int stem_writeback_rows(const stem_shape_t* shape, const void* dE_rows, const in
                         int32_t* host_n, void* stream);
 
 /*
+ * The same write-back through the GPU's copy engine, for callers that know the row count on
+ * the host (n_rows, a value): two asynchronous device-to-host copies on `stream`,
+ * host_rows[0:n_rows,:] and host_ids[0:n_rows].  Prefer it when the write-back overlaps other
+ * kernels: stores issued by SM code that saturate the host link's outbound direction also
+ * delay the GPU's own command fetch over that link, and with it every kernel launched
+ * meanwhile; copy-engine traffic does not.  A caller that pipelines layers can read
+ * *n_unique back one layer ahead without draining the GPU.
+ */
+int stem_writeback_rows_dma(const stem_shape_t* shape, const void* dE_rows, const int32_t* unique_ids,
+                            int32_t n_rows, void* host_rows, int32_t* host_ids, void* stream);
+
+/*
  * Plain contraction on the same tensor-core kernel the layer uses (the y = H W_down^T
  * step is exactly this; exposed for testing and reuse):
  *   C[m,n] = sum_k A(m,k) B(n,k),  C row-major [M,N] (bf16 if c_fp32 == 0, else fp32).

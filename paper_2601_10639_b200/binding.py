@@ -28,7 +28,7 @@ FLAG_SINGLE_CTA = 2
 EXPORTS = (
     "stem_version", "stem_status_string", "stem_workspace_bytes", "stem_init_workspace",
     "stem_query_status", "stem_dedup_ids", "stem_ffn_forward", "stem_ffn_backward",
-    "stem_prefetch_rows", "stem_writeback_rows", "stem_gemm_bf16", "stem_step_arena_bytes",
+    "stem_prefetch_rows", "stem_writeback_rows", "stem_writeback_rows_dma", "stem_gemm_bf16", "stem_step_arena_bytes",
     "stem_ffn_step_host", "stem_ffn_step_host_flush", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
     "stem_dedup_ids_static", "stem_dedup_static_max_tokens",
 )
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
             "stem_ffn_backward": [shp] + [vp] * 17 + [sz, vp],
             "stem_prefetch_rows": [shp, vp, vp, vp, vp, vp, vp],
             "stem_writeback_rows": [shp, vp, vp, vp, vp, vp, vp, vp],
+            "stem_writeback_rows_dma": [shp, vp, vp, i32, vp, vp, vp],
             "stem_gemm_bf16": [i32, i32, i32, vp, i32, vp, i32, vp, i32, i32, vp, vp],
             "stem_step_arena_bytes": [shp, ctypes.POINTER(sz)],
             "stem_dedup_ids_static": [shp, vp, vp, vp, vp, vp, vp, vp, vp],
@@ -168,6 +169,11 @@ def stem_prefetch_rows(shape, ids, n_ids, table, dev_cache, ws, stream=None) -> 
 def stem_writeback_rows(shape, dE_rows, unique_ids, n_rows, host_rows, host_ids, host_n, stream=None) -> None:
     _check(lib().stem_writeback_rows(ctypes.byref(shape), _p(dE_rows), _p(unique_ids), _p(n_rows), _p(host_rows),
                                      _p(host_ids), _p(host_n), _stream(stream)), "stem_writeback_rows")
+
+
+def stem_writeback_rows_dma(shape, dE_rows, unique_ids, n_rows: int, host_rows, host_ids, stream=None) -> None:
+    _check(lib().stem_writeback_rows_dma(ctypes.byref(shape), _p(dE_rows), _p(unique_ids), int(n_rows), _p(host_rows),
+                                         _p(host_ids), _stream(stream)), "stem_writeback_rows_dma")
 
 
 def stem_gemm_bf16(M, N, K, A, a_mn, B, b_mn, C, c_fp32, flags, ws, stream=None) -> None:

@@ -136,11 +136,12 @@ cudaError_t gemm(const stem_shape_t* s, int M, int N, int K, const void* A, bool
   return launch_simt_gemm(s->dtype, M, N, K, A, a_mn, B, b_mn, kind, ep, st);
 }
 
-int pinned_or_device(const void* p, const void** dev_ptr) {
+int pinned_or_device(const void* p, const void** dev_ptr, bool* on_host = nullptr) {
   cudaPointerAttributes attr;
   if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_NOT_PINNED; }
   if (attr.type == cudaMemoryTypeUnregistered) return STEM_ERR_NOT_PINNED;
   *dev_ptr = attr.devicePointer ? attr.devicePointer : p;
+  if (on_host) *on_host = attr.type == cudaMemoryTypeHost;
   return STEM_OK;
 }
 
@@ -310,11 +311,12 @@ int stem_prefetch_rows(const stem_shape_t* shape, const int32_t* ids, const int3
   if (shape->T == 0) return STEM_OK;
   if (!ids || !n_ids || !table || !dev_cache || !aligned16(table) || !aligned16(dev_cache)) return STEM_ERR_INVALID_ARG;
   const void* src = nullptr;
-  if (int rc = pinned_or_device(table, &src)) return rc;
+  bool on_host = false;
+  if (int rc = pinned_or_device(table, &src, &on_host)) return rc;
   const int max_rows = shape->T < shape->V ? shape->T : shape->V;
   const size_t row_bytes = static_cast<size_t>(shape->d_ff) * elem_bytes(shape->dtype);
   ProfScope prof("prefetch_rows", static_cast<cudaStream_t>(stream));
-  cudaError_t e = launch_gather_rows(max_rows, shape->V, row_bytes, ids, n_ids, src, dev_cache,
+  cudaError_t e = launch_gather_rows(max_rows, shape->V, row_bytes, ids, n_ids, src, on_host, dev_cache,
                                      ws ? status_of(ws) : nullptr, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
 }
@@ -337,6 +339,25 @@ int stem_writeback_rows(const stem_shape_t* shape, const void* dE_rows, const in
   cudaError_t e = launch_writeback_rows(max_rows, row_bytes, dE_rows, unique_ids, n_rows, const_cast<void*>(hr),
                                         static_cast<int32_t*>(const_cast<void*>(hi)),
                                         static_cast<int32_t*>(const_cast<void*>(hn)), static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
+int stem_writeback_rows_dma(const stem_shape_t* shape, const void* dE_rows, const int32_t* unique_ids,
+                            int32_t n_rows, void* host_rows, int32_t* host_ids, void* stream) {
+  if (int rc = check_shape(shape)) return rc;
+  const int max_rows = shape->T < shape->V ? shape->T : shape->V;
+  if (n_rows < 0 || n_rows > max_rows) return STEM_ERR_INVALID_ARG;
+  if (n_rows == 0) return STEM_OK;
+  if (!dE_rows || !unique_ids || !host_rows || !host_ids) return STEM_ERR_INVALID_ARG;
+  const void* unused = nullptr;
+  if (int rc = pinned_or_device(host_rows, &unused)) return rc;
+  if (int rc = pinned_or_device(host_ids, &unused)) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t row_bytes = static_cast<size_t>(shape->d_ff) * elem_bytes(shape->grad_dtype);
+  ProfScope prof("writeback_rows", st);
+  cudaError_t e = cudaMemcpyAsync(host_rows, dE_rows, row_bytes * n_rows, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(host_ids, unique_ids, sizeof(int32_t) * static_cast<size_t>(n_rows), cudaMemcpyDeviceToHost, st);
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
 }
 

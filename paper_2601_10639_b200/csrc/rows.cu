@@ -2,13 +2,21 @@
 // (cache[r] = table[ids[r]]) and the gradient write-back.  Row counts are device scalars,
 // so the grids are sized for the upper bound and CTAs stride over the real count.
 // 16-byte accesses, one row spread across the CTA; when the table is page-locked host
-// memory the loads cross the host link directly (no staging copy).
+// memory the loads cross the host link directly (no staging copy).  Kernels that talk to
+// host memory are meant to run beside the contraction kernels of another layer, which hold
+// every SM with one large CTA each: they are launched as kHostLinkCtas CTAs of
+// kHostLinkThreads threads.  Even two of those fit next to a contraction CTA (registers,
+// threads; no shared memory), so the contraction never waits for an SM, and eight 16-byte
+// loads in flight per thread still cover several times the host link's bandwidth-delay
+// product.
 #include "stem_internal.h"
 
 namespace stem {
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;          // device-to-device gathers
+constexpr int kHostLinkCtas = 32;
+constexpr int kHostLinkThreads = 128;
 
 __global__ void __launch_bounds__(kThreads)
 gather_rows_kernel(int V, int vec_per_row, const int32_t* __restrict__ ids,
@@ -16,8 +24,8 @@ gather_rows_kernel(int V, int vec_per_row, const int32_t* __restrict__ ids,
                    uint4* __restrict__ dst, int32_t* status) {
   const int n = *n_ids;
   // a CTA handles `rows_per_cta` rows per step so short rows still fill the block
-  const int lanes_per_row = min(vec_per_row, kThreads);
-  const int rows_per_cta = kThreads / lanes_per_row;
+  const int lanes_per_row = min(vec_per_row, static_cast<int>(blockDim.x));
+  const int rows_per_cta = static_cast<int>(blockDim.x) / lanes_per_row;
   const int sub = threadIdx.x / lanes_per_row, lane = threadIdx.x % lanes_per_row;
   if (sub >= rows_per_cta) return;
   for (int r = blockIdx.x * rows_per_cta + sub; r < n; r += gridDim.x * rows_per_cta) {
@@ -29,6 +37,13 @@ gather_rows_kernel(int V, int vec_per_row, const int32_t* __restrict__ ids,
     const uint4* src = table + static_cast<size_t>(id) * vec_per_row;
     uint4* out = dst + static_cast<size_t>(r) * vec_per_row;
     int c = lane;
+    for (; c + 7 * lanes_per_row < vec_per_row; c += 8 * lanes_per_row) {
+      uint4 a[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) a[j] = src[c + j * lanes_per_row];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) out[c + j * lanes_per_row] = a[j];
+    }
     for (; c + 3 * lanes_per_row < vec_per_row; c += 4 * lanes_per_row) {
       const uint4 a0 = src[c], a1 = src[c + lanes_per_row], a2 = src[c + 2 * lanes_per_row],
                   a3 = src[c + 3 * lanes_per_row];
@@ -39,34 +54,50 @@ gather_rows_kernel(int V, int vec_per_row, const int32_t* __restrict__ ids,
   }
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kHostLinkThreads)
 writeback_rows_kernel(int vec_per_row, const uint4* __restrict__ rows,
                       const int32_t* __restrict__ unique_ids, const int32_t* __restrict__ n_rows,
                       uint4* __restrict__ host_rows, int32_t* __restrict__ host_ids,
                       int32_t* __restrict__ host_n) {
   const int n = *n_rows;
   const size_t total = static_cast<size_t>(n) * vec_per_row;
-  const size_t stride = static_cast<size_t>(gridDim.x) * kThreads;
-  for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < total; i += stride)
-    host_rows[i] = rows[i];
-  for (size_t i = static_cast<size_t>(blockIdx.x) * kThreads + threadIdx.x; i < static_cast<size_t>(n); i += stride)
-    host_ids[i] = unique_ids[i];
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  for (; i + 3 * stride < total; i += 4 * stride) {   // four loads in flight per thread
+    const uint4 a0 = rows[i], a1 = rows[i + stride], a2 = rows[i + 2 * stride], a3 = rows[i + 3 * stride];
+    host_rows[i] = a0; host_rows[i + stride] = a1; host_rows[i + 2 * stride] = a2; host_rows[i + 3 * stride] = a3;
+  }
+  for (; i < total; i += stride) host_rows[i] = rows[i];
+  for (size_t j = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < static_cast<size_t>(n); j += stride)
+    host_ids[j] = unique_ids[j];
   if (blockIdx.x == 0 && threadIdx.x == 0) *host_n = n;
+}
+
+// An SM cannot hold CTAs of two kernels that run under different shared-memory / L1 splits,
+// and the contraction kernels need the largest shared-memory split.  Asking for the same
+// split here (these kernels use no shared memory themselves) lets their CTAs share an SM
+// with a contraction CTA instead of waiting for it, or making it wait.
+template <typename Kernel>
+cudaError_t prefer_max_shared(Kernel kernel) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
 }
 
 }  // namespace
 
 cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int32_t* ids,
-                               const int32_t* n_ids, const void* table, void* dst,
+                               const int32_t* n_ids, const void* table, bool table_on_host, void* dst,
                                int32_t* status, cudaStream_t stream) {
   if (max_rows <= 0) return cudaSuccess;
   const int vec = static_cast<int>(row_bytes / 16);
-  const int lanes_per_row = vec < kThreads ? vec : kThreads;
-  const int rows_per_cta = kThreads / lanes_per_row;
+  const int threads = table_on_host ? kHostLinkThreads : kThreads;
+  const int lanes_per_row = vec < threads ? vec : threads;
+  const int rows_per_cta = threads / lanes_per_row;
   int blocks = (max_rows + rows_per_cta - 1) / rows_per_cta;
-  const int cap = device_sm_count() * 8;
+  const int cap = table_on_host ? kHostLinkCtas : device_sm_count() * 8;
   if (blocks > cap) blocks = cap;
-  gather_rows_kernel<<<blocks, kThreads, 0, stream>>>(V, vec, ids, n_ids, static_cast<const uint4*>(table),
+  static const cudaError_t configured = prefer_max_shared(gather_rows_kernel);
+  if (configured != cudaSuccess) return configured;
+  gather_rows_kernel<<<blocks, threads, 0, stream>>>(V, vec, ids, n_ids, static_cast<const uint4*>(table),
                                                      static_cast<uint4*>(dst), status);
   count_launches(1);
   return cudaGetLastError();
@@ -77,8 +108,10 @@ cudaError_t launch_writeback_rows(int max_rows, size_t row_bytes, const void* ro
                                   int32_t* host_ids, int32_t* host_n, cudaStream_t stream) {
   if (max_rows <= 0) return cudaSuccess;
   const int vec = static_cast<int>(row_bytes / 16);
-  const int blocks = device_sm_count() * 4;
-  writeback_rows_kernel<<<blocks, kThreads, 0, stream>>>(vec, static_cast<const uint4*>(rows), unique_ids,
+  const int blocks = kHostLinkCtas;
+  static const cudaError_t configured = prefer_max_shared(writeback_rows_kernel);
+  if (configured != cudaSuccess) return configured;
+  writeback_rows_kernel<<<blocks, kHostLinkThreads, 0, stream>>>(vec, static_cast<const uint4*>(rows), unique_ids,
                                                         n_rows, static_cast<uint4*>(host_rows), host_ids, host_n);
   count_launches(1);
   return cudaGetLastError();
