@@ -166,6 +166,121 @@ def run_reference(args, w):
     }))
 
 
+def run_host_stack(args, w):
+    """Workload with the tables of a stack of independent layers in pinned host memory: a step is
+    forward + backward of every layer, rows prefetched and gradient rows written back on side
+    streams.  Reports tokens/s (all layers) and the exposed copy time: the time of the same stack
+    with device-resident tables subtracted from the host-table time."""
+    import torch
+    from paper_2601_10639_b200 import binding as B
+    from paper_2601_10639_b200 import runner
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    B.lib()
+    dt = torch.bfloat16
+    T, d, F, V, L = (args.tokens or w.T), w.d_model, w.d_ff, w.V, w.layers
+    gcode = B.DTYPE_BF16 if args.grad_bf16 else B.DTYPE_FP32
+    gen = torch.Generator(device=dev).manual_seed(args.seed)
+    shape = B.make_shape(T, d, F, V, B.DTYPE_BF16, gcode, 0)
+    W_gate = (torch.randn(F, d, generator=gen, device=dev) * d ** -0.5).to(dt)
+    W_down = (torch.randn(d, F, generator=gen, device=dev) * F ** -0.5).to(dt)
+    xs = [torch.randn(T, d, generator=gen, device=dev).to(dt) for _ in range(L)]
+    dys = [torch.randn(T, d, generator=gen, device=dev).to(dt) for _ in range(L)]
+    idss = [torch.from_numpy(synth.token_ids(args.seed, T, V, w.id_dist, layer=l)).to(dev) for l in range(L)]
+    dev_tables, host_tables = [], []
+    for l in range(L):
+        E = torch.empty(V, F, device=dev, dtype=dt)
+        for r0 in range(0, V, 4096):
+            r1 = min(V, r0 + 4096)
+            E[r0:r1] = (torch.randn(r1 - r0, F, generator=gen, device=dev) * 0.02).to(dt)
+        dev_tables.append(E)
+        h = torch.empty(V, F, dtype=dt).pin_memory()
+        h.copy_(E)
+        host_tables.append(h)
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+    results = {}
+    for name, resident in (("resident", True), ("host", False)):
+        stack = runner.HostTableStack(shape, L, dev_tables if resident else host_tables, W_gate, W_down, resident)
+        for _ in range(args.warmup):
+            stack.step(xs, idss, dys)
+        stack.finish()
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = B.stem_launch_count()
+        with ClockSampler(0) as clocks:
+            t0 = time.time()
+            ev0.record(stream)
+            for _ in range(args.steps):
+                stack.step(xs, idss, dys)
+            stack.finish()
+            ev1.record(stream)
+            torch.cuda.synchronize()
+            t1 = time.time()
+        assert B.stem_query_status(stack.ws) == B.OK
+        results[name] = {"ms": ev0.elapsed_time(ev1) / args.steps, "launches": B.stem_launch_count() - l0,
+                         "clocks": clocks.summary(t0, t1),
+                         "n_unique": [int(k["n_unique"].item()) for k in stack.slots]}
+        if not resident:
+            k = stack.slots[(L - 1) % 3]
+            n = int(k["host_n"][0])
+            assert n == int(k["n_unique"].item())
+            assert torch.equal(k["host_rows"][:n], k["dE_rows"][:n].cpu())      # what reached the host is the gradient
+        del stack
+
+    # ---- the host link by itself: plain pinned copies (the denominator), then the row movers alone
+    def timed(fn, n=5):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+    nbytes = 256 << 20
+    hbuf = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    dbuf = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    link = {"h2d_gbs": nbytes / timed(lambda: dbuf.copy_(hbuf, non_blocking=True)) / 1e6,
+            "d2h_gbs": nbytes / timed(lambda: hbuf.copy_(dbuf, non_blocking=True)) / 1e6}
+    probe = runner.HostTableStack(shape, L, host_tables, W_gate, W_down, False)
+    k = probe.slots[0]
+    B.stem_dedup_ids(shape, idss[0], k["unique_ids"], k["n_unique"], k["inverse"], k["perm"], k["seg_offsets"], probe.ws)
+    n0 = int(k["n_unique"].item())
+    gsz = 2 if args.grad_bf16 else 4
+    t_pf = timed(lambda: B.stem_prefetch_rows(shape, k["unique_ids"], k["n_unique"], host_tables[0], k["cache"], probe.ws))
+    t_wb = timed(lambda: B.stem_writeback_rows(shape, k["dE_rows"], k["unique_ids"], k["n_unique"], k["host_rows"],
+                                               k["host_ids"], k["host_n"]))
+    t_dma = timed(lambda: B.stem_writeback_rows_dma(shape, k["dE_rows"], k["unique_ids"], n0, k["host_rows"], k["host_ids"]))
+    link.update(prefetch_rows_gbs=n0 * F * 2 / t_pf / 1e6, writeback_rows_kernel_gbs=n0 * F * gsz / t_wb / 1e6,
+                writeback_rows_dma_gbs=n0 * F * gsz / t_dma / 1e6, prefetch_rows_ms=t_pf, writeback_rows_dma_ms=t_dma)
+    del probe
+    host_ms, res_ms = results["host"]["ms"], results["resident"]["ms"]
+    n_u = float(np.mean(results["host"]["n_unique"]))
+    peaks = load_peaks()
+    tf = 12.0 * L * T * d * F / (host_ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": METRIC, "value": L * T / (host_ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": host_ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "layers": L, "T": T, "d_model": d, "d_ff": F, "V": V, "ids": w.id_dist,
+                   "tables": "pinned host memory, one per layer", "grad_dtype": "bf16" if args.grad_bf16 else "f32",
+                   "l2": "working set exceeds L2; no flush"},
+        "gpu_launches": int(results["host"]["launches"]), "clocks": results["host"]["clocks"], "tflops_step": tf,
+        "host_tables": {"ms_per_step": host_ms, "ms_per_layer": host_ms / L},
+        "device_tables": {"ms_per_step": res_ms, "ms_per_layer": res_ms / L, "clocks": results["resident"]["clocks"]},
+        "exposed_copy_ms_per_step": host_ms - res_ms, "exposed_copy_ms_per_layer": (host_ms - res_ms) / L,
+        "host_link": link, "rows_prefetched_per_layer": n_u, "prefetch_bytes_per_layer": n_u * F * 2,
+        "writeback_bytes_per_layer": n_u * F * gsz,
+        "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": tf / peaks["bf16_tflops_sustained"], "traffic": None,
+                     "peak_source": peaks["source"] + " (sustained bf16 GEMM, of measured)",
+                     "kernel": "whole step (six contractions per layer)"},
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -178,6 +293,7 @@ def main():
     ap.add_argument("--seed", type=int, default=synth.BASE_SEED)
     ap.add_argument("--tokens", type=int, default=0,
                     help="override the workload's token count (small cases for profiler captures; not a bench line)")
+    ap.add_argument("--grad-bf16", action="store_true", help="host-table workload: bf16 weight and table gradients")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
@@ -186,6 +302,12 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, w)
+        return
+
+    if w.host_tables:
+        if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+            raise SystemExit("the host-table workload is a one-GPU measurement")
+        run_host_stack(args, w)
         return
 
     import torch

@@ -103,3 +103,116 @@ def state_from_numpy(inputs: dict, dtype_code: int, V: int, grad_dtype: int = B.
     st.E = to_device(inputs["E"], dtype_code, device)
     st.ids = to_device(inputs["ids"], dtype_code, device)
     return st.allocate(backward)
+
+
+class HostTableStack:
+    """A stack of independent STEM layers whose tables live in page-locked host memory
+    (paper Section 3.4: tables offloaded to CPU, the rows of the deduplicated ids prefetched
+    asynchronously with layer compute; Table 1 notes: table gradients go back to the CPU).
+
+    Stream choreography per layer l (ids of every layer are known up front):
+
+        main stream   dedup(l+1) | wait rows(l) | forward(l) backward(l) on the row cache
+        fetch stream              rows(l+1) = table_{l+1}[unique_ids(l+1)]   (over the host link)
+        write stream                                          dE rows(l) -> host (copy engine)
+
+    so the row prefetch of layer l+1 and the gradient write-back of layer l-1 run under the
+    GEMMs of layer l.  Index arrays, row caches and gradient-row buffers rotate through three
+    slots: while layer l computes, slot l+1 is being filled and slot l-1 is being written back.
+    The write-back uses the copy engine, which needs the row count on the host: n_unique of
+    layer l is copied back right after dedup(l), a full layer before it is needed, so reading
+    it never drains the GPU's queue.  With ``resident=True`` the tables are device tensors and
+    the layers read them directly (no prefetch, no write-back): the reference against which
+    exposed copy time is measured.  All arithmetic and every copy is a libstem call (plus the
+    4-byte count read); this class only orders them.
+    """
+
+    def __init__(self, shape: B.StemShape, layers: int, tables, W_gate, W_down, resident: bool, device="cuda"):
+        self.shape, self.layers, self.tables, self.resident = shape, layers, tables, resident
+        self.W_gate, self.W_down = W_gate, W_down
+        s = shape
+        T, d, F = s.T, s.d_model, s.d_ff
+        dt, gdt = torch_dtype(s.dtype), torch_dtype(s.grad_dtype)
+        R = max(min(T, s.V), 1)
+        self.R = R
+        self.cache_shape = B.make_shape(T, d, F, R, s.dtype, s.grad_dtype, s.flags)
+        self.main = torch.cuda.current_stream()
+        self.fetch, self.write = torch.cuda.Stream(), torch.cuda.Stream()
+        self.ws = torch.empty(max(B.stem_workspace_bytes(s), 256), dtype=torch.uint8, device=device)
+        B.stem_init_workspace(self.ws)
+        self.y = torch.empty(T, d, dtype=dt, device=device)
+        self.dx = torch.empty(T, d, dtype=dt, device=device)
+        self.G = torch.empty(T, F, dtype=dt, device=device)
+        self.H = torch.empty(T, F, dtype=dt, device=device)
+        self.dW_gate = torch.empty(F, d, dtype=gdt, device=device)
+        self.dW_down = torch.empty(d, F, dtype=gdt, device=device)
+        self.slots = []
+        for _ in range(3):
+            slot = {
+                "unique_ids": torch.empty(R, dtype=torch.int32, device=device),
+                "n_unique": torch.zeros(1, dtype=torch.int32, device=device),
+                "inverse": torch.empty(T, dtype=torch.int32, device=device),
+                "perm": torch.empty(T, dtype=torch.int32, device=device),
+                "seg_offsets": torch.empty(R + 1, dtype=torch.int32, device=device),
+                "dE_rows": torch.empty(R, F, dtype=gdt, device=device),
+                "deduped": torch.cuda.Event(), "fetched": torch.cuda.Event(), "bwd_done": torch.cuda.Event(),
+                "written": torch.cuda.Event(), "counted": torch.cuda.Event(), "used": False,
+            }
+            if not resident:
+                slot["cache"] = torch.empty(R, F, dtype=dt, device=device)
+                slot["host_rows"] = torch.empty(R, F, dtype=gdt).pin_memory()
+                slot["host_ids"] = torch.empty(R, dtype=torch.int32).pin_memory()
+                slot["host_n"] = torch.zeros(1, dtype=torch.int32).pin_memory()
+            self.slots.append(slot)
+
+    def _dedup_and_fetch(self, l: int, ids):
+        k = self.slots[l % 3]
+        if k["used"] and not self.resident:
+            # the slot's index arrays and gradient rows may still be in use by layer l-3's write-back
+            self.main.wait_event(k["written"])
+        B.stem_dedup_ids(self.shape, ids, k["unique_ids"], k["n_unique"], k["inverse"], k["perm"], k["seg_offsets"],
+                         self.ws, self.main)
+        if self.resident:
+            return
+        k["deduped"].record(self.main)
+        self.fetch.wait_event(k["deduped"])
+        with torch.cuda.stream(self.fetch):
+            k["host_n"].copy_(k["n_unique"], non_blocking=True)     # the row count, one layer ahead of its use
+        k["counted"].record(self.fetch)
+        B.stem_prefetch_rows(self.shape, k["unique_ids"], k["n_unique"], self.tables[l], k["cache"], self.ws, self.fetch)
+        k["fetched"].record(self.fetch)
+
+    def step(self, xs, idss, dys, on_layer=None):
+        """One forward + backward of every layer.  xs, idss, dys: per-layer device tensors."""
+        self._dedup_and_fetch(0, idss[0])
+        for l in range(self.layers):
+            if l + 1 < self.layers:
+                self._dedup_and_fetch(l + 1, idss[l + 1])
+            k = self.slots[l % 3]
+            if self.resident:
+                shape, ids, E = self.shape, idss[l], self.tables[l]
+            else:
+                self.main.wait_event(k["fetched"])
+                shape, ids, E = self.cache_shape, k["inverse"], k["cache"]
+            B.stem_ffn_forward(shape, xs[l], ids, self.W_gate, E, self.W_down, self.y, self.G, self.H, self.ws, self.main)
+            B.stem_ffn_backward(shape, dys[l], xs[l], ids, self.W_gate, E, self.W_down, self.G, self.H, k["perm"],
+                                k["seg_offsets"], k["n_unique"], self.dx, self.dW_gate, self.dW_down, k["dE_rows"],
+                                k["unique_ids"], self.ws, self.main)
+            k["bwd_done"].record(self.main)
+            k["used"] = True
+            if not self.resident:
+                k["counted"].synchronize()      # dedup(l) finished a layer ago: no stall in steady state
+                n_u = int(k["host_n"][0])
+                self.write.wait_event(k["bwd_done"])
+                B.stem_writeback_rows_dma(self.shape, k["dE_rows"], k["unique_ids"], n_u, k["host_rows"], k["host_ids"],
+                                          self.write)
+                k["written"].record(self.write)
+            if on_layer is not None:
+                on_layer(l, k)
+
+    def finish(self):
+        """Make the main stream wait for the outstanding write-backs."""
+        if not self.resident:
+            for k in self.slots:
+                if k["used"]:
+                    self.main.wait_event(k["written"])
