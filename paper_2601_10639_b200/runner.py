@@ -182,12 +182,33 @@ class HostTableStack:
         B.stem_prefetch_rows(self.shape, k["unique_ids"], k["n_unique"], self.tables[l], k["cache"], self.ws, self.fetch)
         k["fetched"].record(self.fetch)
 
+    def _writeback(self, l: int, after=None):
+        k = self.slots[l % 3]
+        k["counted"].synchronize()          # dedup(l) finished more than a layer ago: no stall in steady state
+        n_u = int(k["host_n"][0])
+        self.write.wait_event(k["bwd_done"])
+        if after is not None:
+            # The 4-byte count read of the layer being prefetched shares the device-to-host copy
+            # engine with this bulk copy; letting it go first keeps the prefetch behind it from
+            # waiting for the whole write-back.
+            self.write.wait_event(after)
+        B.stem_writeback_rows_dma(self.shape, k["dE_rows"], k["unique_ids"], n_u, k["host_rows"], k["host_ids"],
+                                  self.write)
+        k["written"].record(self.write)
+
     def step(self, xs, idss, dys, on_layer=None):
-        """One forward + backward of every layer.  xs, idss, dys: per-layer device tensors."""
+        """One forward + backward of every layer.  xs, idss, dys: per-layer device tensors.
+        on_layer(l, slot) is called once layer l's work (write-back included) has been enqueued."""
         self._dedup_and_fetch(0, idss[0])
         for l in range(self.layers):
+            nxt = None
             if l + 1 < self.layers:
                 self._dedup_and_fetch(l + 1, idss[l + 1])
+                nxt = self.slots[(l + 1) % 3]
+            if l > 0 and not self.resident:
+                self._writeback(l - 1, after=nxt["counted"] if nxt is not None else None)
+            if l > 0 and on_layer is not None:
+                on_layer(l - 1, self.slots[(l - 1) % 3])
             k = self.slots[l % 3]
             if self.resident:
                 shape, ids, E = self.shape, idss[l], self.tables[l]
@@ -200,15 +221,11 @@ class HostTableStack:
                                 k["unique_ids"], self.ws, self.main)
             k["bwd_done"].record(self.main)
             k["used"] = True
-            if not self.resident:
-                k["counted"].synchronize()      # dedup(l) finished a layer ago: no stall in steady state
-                n_u = int(k["host_n"][0])
-                self.write.wait_event(k["bwd_done"])
-                B.stem_writeback_rows_dma(self.shape, k["dE_rows"], k["unique_ids"], n_u, k["host_rows"], k["host_ids"],
-                                          self.write)
-                k["written"].record(self.write)
-            if on_layer is not None:
-                on_layer(l, k)
+        last = self.layers - 1
+        if not self.resident:
+            self._writeback(last)
+        if on_layer is not None:
+            on_layer(last, self.slots[last % 3])
 
     def finish(self):
         """Make the main stream wait for the outstanding write-backs."""
