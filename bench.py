@@ -32,6 +32,20 @@ METRIC = "STEM-FFN fwd+bwd tokens/sec (1B-class layer, dedup + forward + backwar
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+def rank_seed(seed: int, rank: int) -> int:
+    """Every rank is an independent replica with its own batch: same shapes, different draws."""
+    return seed + rank
+
+
+def max_over_ranks(values, device):
+    """Element-wise maximum over the ranks of a list of floats (multi-GPU times are the slowest rank's)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -341,7 +355,7 @@ def main():
     for r0 in range(0, V, 4096):
         r1 = min(V, r0 + 4096)
         st.E[r0:r1] = (torch.randn(r1 - r0, F, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(dt)
-    ids_np = synth.token_ids(args.seed + rank, T, V, w.id_dist)
+    ids_np = synth.token_ids(rank_seed(args.seed, rank), T, V, w.id_dist)
     st.ids = torch.from_numpy(ids_np).to(dev)
     st.allocate(backward)
     stream = torch.cuda.current_stream()
@@ -411,11 +425,10 @@ def main():
 
     # ---- max over ranks ------------------------------------------------------------------------
     if world > 1:
-        t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t[0])
+        t = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0], dev)
+        ms_total = t[0]
         if e2e:
-            e2e["ms"] = float(t[1])
+            e2e["ms"] = t[1]
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
