@@ -1,25 +1,24 @@
 // Table-gradient reduce: dE_rows[r,:] = sum over the positions p of segment r of
 // dU[perm[p],:], in a fixed order, without floating-point atomics.
 //
-// The sorted position range [0,T) is cut into blocks of kSegBlk positions.  Pass 1: one CTA
-// per (block, column slab) walks its positions in order, accumulating in fp32 registers.
-// A run whose segment lies wholly inside the block is final and is written to dE_rows; a
-// run whose segment crosses a block edge (at most the first and the last run of a block)
-// goes to a partial row, and every block records which segment (if any) starts inside it and
-// runs past its end.  Pass 2: the CTAs of such a block add that segment's partial rows; the
-// others exit at once.  Every summation order depends on the index arrays only, so the
-// result is bitwise reproducible.  HBM-bound: every dU row is read once with 16-byte loads,
-// coalesced along d_ff.
+// The sorted position range [0,T) is cut into blocks of at most kSegBlk positions.  One CTA per
+// (block, column slab) walks its positions in order, accumulating in fp32 registers.  A run
+// whose segment lies wholly inside the block is final and is written to dE_rows; a run whose
+// segment crosses a block edge (at most the first and the last run of a block) goes to a
+// partial row.  The CTAs that hold parts of such a segment count themselves off on an
+// integer counter; the one that arrives last adds the segment's partial rows in block order
+// and writes the row.  Which CTA that is varies from run to run, the order of the additions
+// does not, so the result is bitwise reproducible.  One launch; HBM-bound: every dU row is
+// read once with 16-byte loads, coalesced along d_ff.
 #include "stem_internal.h"
 
 namespace stem {
 namespace {
 
-constexpr int kSegBlk = 64;     // sorted positions per CTA of pass 1
+constexpr int kSegBlk = 64;     // most sorted positions per CTA (the launch picks blk_len <= kSegBlk)
+constexpr int kCtasPerSm = 7;   // register budget the kernel is compiled for
 constexpr int kThreads = 128;   // pass 1: one thread per vector of columns
 constexpr int kBatch = 8;       // rows requested before the first is consumed
-constexpr int kRowLanes = 8;    // pass 2: partial rows summed side by side
-constexpr int kColLanes = 32;
 
 template <typename T> struct Vec;
 template <> struct Vec<float> {
@@ -62,26 +61,27 @@ __device__ __forceinline__ void store_row(TOut* dst, const float (&v)[VI]) {
   for (int i = 0; i < VI; i += Vec<TOut>::N) Vec<TOut>::store(dst + i, v + i);
 }
 
-// Scratch layout: cross_seg[n_blk] (segment that starts in the block and crosses its end, or
-// -1), then 2 partial rows per block.
-__host__ __device__ inline size_t partial_offset_bytes(int n_blk) {
-  return (static_cast<size_t>(n_blk) * 4 + 255) / 256 * 256;
+// Scratch layout: arrival counters [n_blk][n_slabs] (one per block in which a crossing
+// segment can start, per column slab; zeroed before each launch), then 2 partial rows per
+// block.
+__host__ __device__ inline size_t partial_offset_bytes(int n_blk, int n_slabs) {
+  return (static_cast<size_t>(n_blk) * n_slabs * 4 + 255) / 256 * 256;
 }
 
 template <typename TIn, typename TOut>
-__global__ void __launch_bounds__(kThreads, 6)
-segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* __restrict__ perm,
-                       const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ n_unique,
-                       TOut* __restrict__ dE_rows, int32_t* __restrict__ cross_seg,
-                       float* __restrict__ partial) {
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+segreduce_kernel(int T, int F, int blk_len, const TIn* __restrict__ dU, const int32_t* __restrict__ perm,
+                 const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ n_unique,
+                 TOut* __restrict__ dE_rows, int32_t* __restrict__ counters, float* partial) {
   constexpr int VI = (Vec<TIn>::N > Vec<TOut>::N) ? Vec<TIn>::N : Vec<TOut>::N;
   constexpr int LD = VI / Vec<TIn>::N;  // 16-byte loads per row per thread
   __shared__ int s_off[kSegBlk + 1];    // offsets of the segments that can touch this block
   __shared__ int s_row[kSegBlk];
   __shared__ int s_loc[kSegBlk];        // position -> index into s_off
+  __shared__ int s_finish[2];           // crossing segments this CTA must finish (index into s_off), or -1
   const int blk = blockIdx.x;
-  const int p0 = blk * kSegBlk;
-  const int cnt = min(kSegBlk, T - p0);
+  const int p0 = blk * blk_len;
+  const int cnt = min(blk_len, T - p0);
   const int n_u = *n_unique;
 
   // r_first = largest r with seg_offsets[r] <= p0, found with kThreads pivots per round
@@ -114,19 +114,14 @@ segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* 
     s_loc[threadIdx.x] = a;
   }
   __syncthreads();
-  if (blockIdx.y == 0 && threadIdx.x == 0) {
-    // a segment that starts in this block and runs past its end is finished by pass 2
-    const int j = s_loc[cnt - 1];
-    cross_seg[blk] = (s_off[j] >= p0 && s_off[j + 1] > p0 + kSegBlk) ? r_first + j : -1;
-  }
   const int col = (blockIdx.y * kThreads + threadIdx.x) * VI;
-  if (col >= F) return;
+  const bool col_ok = col < F;
 
   float acc[VI];
 #pragma unroll
   for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
   bool first_run = true;
-  for (int b0 = 0; b0 < cnt; b0 += kBatch) {
+  for (int b0 = 0; col_ok && b0 < cnt; b0 += kBatch) {
     uint4 raw[kBatch][LD];
 #pragma unroll
     for (int j = 0; j < kBatch; ++j) {
@@ -145,7 +140,7 @@ segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* 
         const int loc = s_loc[q];
         const bool run_ends = (q + 1 == cnt) || (s_loc[q + 1] != loc);
         if (run_ends) {
-          const bool whole = s_off[loc] >= p0 && s_off[loc + 1] <= p0 + kSegBlk;
+          const bool whole = s_off[loc] >= p0 && s_off[loc + 1] <= p0 + blk_len;
           if (whole) {
             store_row<VI, TOut>(dE_rows + static_cast<size_t>(r_first + loc) * F + col, acc);
           } else {
@@ -158,50 +153,49 @@ segreduce_pass1_kernel(int T, int F, const TIn* __restrict__ dU, const int32_t* 
       }
     }
   }
-}
 
-// One CTA per (block, 32 x VI columns); only blocks in which a crossing segment starts do
-// work: kRowLanes partial rows are added side by side, each lane walking its rows in block
-// order, then the lanes are combined in lane order.
-template <typename TOut, int VI>
-__global__ void __launch_bounds__(kRowLanes * kColLanes, 4)
-segreduce_pass2_kernel(int T, int F, const int32_t* __restrict__ seg_offsets,
-                       const int32_t* __restrict__ cross_seg, const float* __restrict__ partial,
-                       TOut* __restrict__ dE_rows) {
-  __shared__ float s_sum[kRowLanes][kColLanes][VI + 1];
-  const int blk = blockIdx.x;
-  const int r = cross_seg[blk];
-  if (r < 0) return;
-  const int cl = threadIdx.x % kColLanes, rl = threadIdx.x / kColLanes;
-  const int col = (blockIdx.y * kColLanes + cl) * VI;
-  const int p0 = blk * kSegBlk;
-  const int seg_begin = seg_offsets[r], seg_end = seg_offsets[r + 1];
-  const int b_last = (seg_end - 1) / kSegBlk;
-  float acc[VI];
+  // ---- crossing segments: the last CTA to arrive adds the parts ----------------------------
+  // At most two per block: the segment of the first position (if it began earlier or runs on)
+  // and that of the last position (if it runs on).  s_off[0] <= p0, so index 0 is the first.
+  __threadfence();   // this CTA's partial rows are visible before it counts itself off
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int n_slabs = gridDim.y;
+    const int j_first = 0, j_last = s_loc[cnt - 1];
+    for (int which = 0; which < 2; ++which) {
+      const int j = which == 0 ? j_first : j_last;
+      int fin = -1;
+      const bool whole = s_off[j] >= p0 && s_off[j + 1] <= p0 + blk_len;
+      if (!whole && !(which == 1 && j_last == j_first)) {
+        const int start_blk = s_off[j] / blk_len, last_blk = (s_off[j + 1] - 1) / blk_len;
+        const int old = atomicAdd(&counters[start_blk * n_slabs + blockIdx.y], 1);
+        if (old == last_blk - start_blk) fin = j;
+      }
+      s_finish[which] = fin;
+    }
+  }
+  __syncthreads();
 #pragma unroll
-  for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
-  if (col < F) {
-    for (int b = blk + rl; b <= b_last; b += kRowLanes) {
+  for (int which = 0; which < 2; ++which) {
+    const int j = s_finish[which];
+    if (j < 0 || !col_ok) continue;
+    __threadfence();   // the other CTAs' partial rows, published before their count, are visible
+    const int seg_begin = s_off[j], seg_end = s_off[j + 1];
+    const int start_blk = seg_begin / blk_len, last_blk = (seg_end - 1) / blk_len;
+#pragma unroll
+    for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
+    for (int b = start_blk; b <= last_blk; ++b) {
       // the segment's run is the first run of block b, unless b is the block it starts in
       // and it does not start at that block's first position
-      const int slot = (b > blk || seg_begin == p0) ? 2 * b : 2 * b + 1;
+      const int slot = (b > start_blk || seg_begin == start_blk * blk_len) ? 2 * b : 2 * b + 1;
       const float* src = partial + static_cast<size_t>(slot) * F + col;
 #pragma unroll
       for (int i = 0; i < VI; i += 4) {
-        const float4 q = *reinterpret_cast<const float4*>(src + i);
+        const float4 q = __ldcg(reinterpret_cast<const float4*>(src + i));
         acc[i] += q.x; acc[i + 1] += q.y; acc[i + 2] += q.z; acc[i + 3] += q.w;
       }
     }
-  }
-#pragma unroll
-  for (int i = 0; i < VI; ++i) s_sum[rl][cl][i] = acc[i];
-  __syncthreads();
-  if (rl == 0 && col < F) {
-#pragma unroll
-    for (int l = 1; l < kRowLanes; ++l)
-#pragma unroll
-      for (int i = 0; i < VI; ++i) acc[i] += s_sum[l][cl][i];
-    store_row<VI, TOut>(dE_rows + static_cast<size_t>(r) * F + col, acc);
+    store_row<VI, TOut>(dE_rows + static_cast<size_t>(r_first + j) * F + col, acc);
   }
 }
 
@@ -209,17 +203,31 @@ template <typename TIn, typename TOut>
 cudaError_t launch_typed(int T, int F, const void* dU, const int32_t* perm, const int32_t* seg_offsets,
                          const int32_t* n_unique, void* dE_rows, void* scratch, cudaStream_t stream) {
   constexpr int VI = (Vec<TIn>::N > Vec<TOut>::N) ? Vec<TIn>::N : Vec<TOut>::N;
-  const int n_blk = (T + kSegBlk - 1) / kSegBlk;
-  int32_t* cross_seg = static_cast<int32_t*>(scratch);
-  float* partial = reinterpret_cast<float*>(static_cast<char*>(scratch) + partial_offset_bytes(n_blk));
-  dim3 grid1(n_blk, (F + kThreads * VI - 1) / (kThreads * VI));
-  segreduce_pass1_kernel<TIn, TOut><<<grid1, kThreads, 0, stream>>>(
-      T, F, static_cast<const TIn*>(dU), perm, seg_offsets, n_unique, static_cast<TOut*>(dE_rows), cross_seg,
-      partial);
-  dim3 grid2(n_blk, (F + kColLanes * VI - 1) / (kColLanes * VI));
-  segreduce_pass2_kernel<TOut, VI><<<grid2, kRowLanes * kColLanes, 0, stream>>>(
-      T, F, seg_offsets, cross_seg, partial, static_cast<TOut*>(dE_rows));
-  count_launches(2);
+  const int n_slabs = (F + kThreads * VI - 1) / (kThreads * VI);
+  // Block length: as long as allowed, then shortened so that the CTAs fill a whole number of
+  // waves of the resident CTA slots (a ragged last wave of full-length blocks costs more than
+  // evenly shorter blocks).
+  static int ctas_per_sm = 0;
+  if (ctas_per_sm == 0) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, segreduce_kernel<TIn, TOut>, kThreads, 0) != cudaSuccess || n < 1)
+      n = 1;
+    ctas_per_sm = n;
+  }
+  const int per_wave = device_sm_count() * ctas_per_sm / n_slabs > 0 ? device_sm_count() * ctas_per_sm / n_slabs : 1;
+  const int min_blk = (T + kSegBlk - 1) / kSegBlk;
+  const int waves = (min_blk + per_wave - 1) / per_wave;
+  int blk_len = (T + waves * per_wave - 1) / (waves * per_wave);
+  if (blk_len < 8) blk_len = 8 < T ? 8 : T;
+  if (blk_len > kSegBlk) blk_len = kSegBlk;
+  const int n_blk = (T + blk_len - 1) / blk_len;
+  int32_t* counters = static_cast<int32_t*>(scratch);
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(scratch) + partial_offset_bytes(n_blk, n_slabs));
+  cudaError_t e = cudaMemsetAsync(counters, 0, static_cast<size_t>(n_blk) * n_slabs * sizeof(int32_t), stream);
+  if (e != cudaSuccess) return e;
+  segreduce_kernel<TIn, TOut><<<dim3(n_blk, n_slabs), kThreads, 0, stream>>>(
+      T, F, blk_len, static_cast<const TIn*>(dU), perm, seg_offsets, n_unique, static_cast<TOut*>(dE_rows), counters, partial);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -227,8 +235,10 @@ cudaError_t launch_typed(int T, int F, const void* dU, const int32_t* perm, cons
 
 size_t segreduce_workspace_bytes(int T, int F) {
   if (T <= 0) return 0;
-  const size_t n_blk = (static_cast<size_t>(T) + kSegBlk - 1) / kSegBlk;
-  return partial_offset_bytes(static_cast<int>(n_blk)) + align_up(2 * n_blk * static_cast<size_t>(F) * sizeof(float), 256);
+  // bounds over every launch shape: blocks of at least 8 positions, the narrowest slab
+  const size_t n_blk = (static_cast<size_t>(T) + 7) / 8;
+  const int n_slabs = (F + kThreads * 4 - 1) / (kThreads * 4);
+  return partial_offset_bytes(static_cast<int>(n_blk), n_slabs) + align_up(2 * n_blk * static_cast<size_t>(F) * sizeof(float), 256);
 }
 
 cudaError_t launch_segreduce(int T, int F, int in_dtype, int out_dtype, const void* dU,
