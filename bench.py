@@ -423,6 +423,25 @@ def main():
         e2e = {"ms": e2e_ms, "h2d": 2 * T * d * esz + T * 4, "d2h": 2 * T * d * esz + 4}
         del arena
 
+    # ---- compact row gather from the device-resident table (the standalone gather figure) ------------
+    gather = None
+    if rank == 0 and dcode == B.DTYPE_BF16:
+        cache = torch.empty(min(T, V), F, dtype=dt, device=dev)
+        b = st.bufs
+        for _ in range(3):
+            B.stem_prefetch_rows(st.shape, b["unique_ids"], b["n_unique"], st.E, cache, b["ws"])
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        g0.record(stream)
+        for _ in range(reps):
+            B.stem_prefetch_rows(st.shape, b["unique_ids"], b["n_unique"], st.E, cache, b["ws"])
+        g1.record(stream)
+        torch.cuda.synchronize()
+        g_ms = g0.elapsed_time(g1) / reps
+        gather = {"rows": n_u, "ms": g_ms, "bytes": 2 * n_u * F * esz}       # rows read once, written once
+        del cache
+
     # ---- max over ranks ------------------------------------------------------------------------
     if world > 1:
         t = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0], dev)
@@ -457,6 +476,14 @@ def main():
             k["gbs"] = seg_bytes / (avg * 1e-3) / 1e9
             k["frac_of_measured_hbm"] = k["gbs"] / peaks["hbm_gbs"]
         kernels[name] = k
+    if gather:
+        gbs = gather["bytes"] / (gather["ms"] * 1e-3) / 1e9
+        kernels["compact_gather"] = {"launch_sets": 20, "avg_ms": gather["ms"], "rows": gather["rows"], "gbs": gbs,
+                                     "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+                                     "note": "cache[r] = E[unique_ids[r]] on the device, back to back, outside the timed step"}
+    if "gate_gemm" in kernels:
+        # rows the fused lookup hands to the epilogue, per second (not a roofline: the kernel is MMA-bound)
+        kernels["gate_gemm"]["fused_lookup_gbs"] = T * F * esz / (kernels["gate_gemm"]["avg_ms"] * 1e-3) / 1e9
     gemms = {n: k for n, k in kernels.items() if n.endswith("_gemm")}
     roofline = None
     if gemms and dcode == B.DTYPE_BF16:
