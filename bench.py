@@ -32,6 +32,13 @@ METRIC = "STEM-FFN fwd+bwd tokens/sec (1B-class layer, dedup + forward + backwar
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+def layer_flops(T: int, d: int, F: int, backward: bool) -> float:
+    """FLOPs (2 per multiply-accumulate) the layer's contractions perform on T tokens: two d x d_ff
+    products per token forward (the up-projection STEM removes is not counted: paper Table 1),
+    and twice that again backward (each forward product has a data and a weight gradient)."""
+    return (12.0 if backward else 4.0) * T * d * F
+
+
 def rank_seed(seed: int, rank: int) -> int:
     """Every rank is an independent replica with its own batch: same shapes, different draws."""
     return seed + rank
@@ -517,7 +524,7 @@ def main():
                    "n_unique": n_u, "backward": backward, "parallelism": f"replicas x{world}",
                    "l2": "per-step working set (~2.5 GB at 1b shapes) exceeds the 126 MB L2; no flush"},
         "gpu_launches": int(launches),
-        "tflops_step": (12.0 if backward else 4.0) * T * d * F / (ms_per_step * 1e-3) / 1e12,
+        "tflops_step": layer_flops(T, d, F, backward) / (ms_per_step * 1e-3) / 1e12,
         "clocks": clock_summary,
         "roofline": roofline,
         "kernels": kernels,

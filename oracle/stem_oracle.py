@@ -21,7 +21,9 @@ Token ids are 0-based.  There are no bias terms (Table 1 caption).
 
 Pins (tests/test_oracle_pins.py): dense SwiGLU on one-hot augmented input through
 torch autograd, central finite differences, brute-force per-id sums and index arrays,
-special values, permutation equivariance.  Every function here has at least one pin.
+special values, permutation equivariance; the two cost-model functions against the
+percentages the paper prints (tests/golden/ffn_saving_fraction.txt).  Every function here
+has at least one pin.
 """
 from __future__ import annotations
 
@@ -137,6 +139,23 @@ def prefetch_rows(unique_ids, n_ids: int, host_E) -> np.ndarray:
     cache[r] = E[unique_ids[r]] for r < n_ids."""
     idx = np.asarray(unique_ids[:n_ids], dtype=np.int64)
     return np.asarray(host_E)[idx].copy()
+
+
+def ffn_macs_per_token(d: int, d_ff: int, stem: bool) -> int:
+    """Multiply-accumulates of one FFN layer per token, forward (Table 1, row "FLOPs", with the
+    element-wise term left out as the paper's text does): three d x d_ff products for a dense
+    SwiGLU block, two for STEM, whose up-projection is a table lookup."""
+    return (2 if stem else 3) * d * d_ff
+
+
+def training_saving_fraction(d: int, d_ff: int, L: int) -> float:
+    """Section 3.2.3, "Training efficiency": per-layer saving of STEM over the dense block,
+    (F_base - F_stem) / F_base with F_base = 4 L d^2 + 2 L^2 d + 3 L d d_ff per sequence and the
+    FFN term 3 -> 2 for STEM.  Written out from the two totals, not from the closed form."""
+    attn = 4 * L * d * d + 2 * L * L * d
+    base = attn + L * ffn_macs_per_token(d, d_ff, stem=False)
+    stem = attn + L * ffn_macs_per_token(d, d_ff, stem=True)
+    return (base - stem) / base
 
 
 def scaled_max_err(got, ref) -> float:

@@ -267,3 +267,47 @@ def test_synth_is_seeded_and_shaped():
     assert 9500 < len(np.unique(mix)) < 11000
     r = synth.round_bf16(a["x"])
     assert np.array_equal(synth.round_bf16(r), r) and np.max(np.abs(r - a["x"]) / np.abs(a["x"])) <= 2.0 ** -8
+
+
+# ---------------------------------------------------------------------------------------
+# cost model: the percentages the paper prints
+# ---------------------------------------------------------------------------------------
+def _golden_rows():
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "ffn_saving_fraction.txt")
+    rows = []
+    for line in open(path):
+        if line.strip() and not line.startswith("#"):
+            name, d, dff, L, pct, ok = line.split()
+            rows.append((name, int(d), int(dff), int(L), float(pct), ok == "1"))
+    return rows
+
+
+def test_saving_fraction_matches_the_printed_percentages():
+    rows = _golden_rows()
+    assert len(rows) == 5
+    for name, d, dff, L, pct, follows in rows:
+        got = 100.0 * O.training_saving_fraction(d, dff, L)
+        closed = 100.0 * dff / (4 * d + 2 * L + 3 * dff)          # the paper's closed form
+        assert abs(got - closed) < 1e-9
+        if follows:
+            assert abs(got - pct) < 0.05, (name, got, pct)        # equal to the printed digit
+        else:
+            assert abs(got - 22.3) < 0.05 and abs(got - pct) > 0.4  # the 3B value is off in the paper
+
+
+def test_flop_accounting_of_the_benchmark():
+    """bench.py counts 2 FLOPs per multiply-accumulate of the two products STEM keeps, and three
+    times the forward count for forward + backward; the checker's forward performs exactly that
+    many multiply-accumulates in its two matrix products."""
+    import bench
+    T, d, F = 7, 12, 20
+    macs = T * O.ffn_macs_per_token(d, F, stem=True)
+    assert O.ffn_macs_per_token(d, F, stem=False) - O.ffn_macs_per_token(d, F, stem=True) == d * F
+    assert bench.layer_flops(T, d, F, backward=False) == 2 * macs
+    assert bench.layer_flops(T, d, F, backward=True) == 3 * 2 * macs
+    x = np.ones((T, d)); Wg = np.ones((F, d)); Wd = np.ones((d, F)); E = np.ones((3, F))
+    _, im = O.forward(x, np.zeros(T, dtype=np.int64), Wg, E, Wd, return_intermediates=True)
+    # with all-ones operands every entry of G is the length of its dot product
+    assert im["G"].shape == (T, F) and float(im["G"][0, 0]) == d
+    assert im["G"].size * d + T * d * F == macs
