@@ -71,6 +71,36 @@ def test_dedup_bit_exact(dist, T, V):
         assert int(st.bufs["unique_ids"][n_u].item()) == -7      # entries past n_u untouched
 
 
+def test_dedup_largest_supported_batch():
+    """T = 2^22 positions (the documented limit), a vocabulary that needs four radix passes."""
+    T, V = 1 << 22, (1 << 30) - 5
+    ids = synth.token_ids(9, T, V, "uniform")                  # all four digits in use
+    ids[T // 2:] = ids[:T // 2][::-1]                           # every id at least twice, far apart
+    ids[::7] = V - 1 - (np.arange(0, T, 7) % 1000)             # and some heavy repeats at the top of the range
+    ref = O.dedup(ids)
+    st = runner.LayerState(B.make_shape(T, 8, 8, V, B.DTYPE_BF16, B.DTYPE_FP32, 0))
+    R = min(T, V)
+    b = st.bufs
+    b["ws"] = torch.empty(B.stem_workspace_bytes(st.shape), dtype=torch.uint8, device="cuda")
+    B.stem_init_workspace(b["ws"])
+    for k, n in (("unique_ids", R), ("n_unique", 1), ("inverse", T), ("perm", T), ("seg_offsets", R + 1)):
+        b[k] = torch.empty(n, dtype=torch.int32, device="cuda")
+    st.ids = torch.from_numpy(ids).cuda()
+    st.dedup()
+    assert st.status() == B.OK
+    n_u = int(b["n_unique"].item())
+    assert n_u == ref["n_unique"]
+    for k, n in (("unique_ids", n_u), ("perm", T), ("seg_offsets", n_u + 1), ("inverse", T)):
+        assert np.array_equal(b[k][:n].cpu().numpy(), ref[k]), k
+
+
+def test_layer_many_tokens_narrow():
+    """A long batch (131072 positions, several hundred row tiles) on a narrow layer: every tile row
+    of the token dimension, ragged d_ff, heavy id repetition."""
+    w = synth.Workload("t", 131072, 64, 136, 5000, "bf16", "zipf")
+    _full_parity(w, synth.make_inputs(w, seed=95), B.DTYPE_BF16, TOL_BF16)
+
+
 def test_dedup_empty_and_bad_ids():
     st = runner.LayerState(B.make_shape(0, 8, 8, 10, B.DTYPE_BF16, B.DTYPE_FP32, 0)).allocate(backward=False)
     st.ids = torch.zeros(1, dtype=torch.int32, device="cuda")
