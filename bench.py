@@ -302,6 +302,38 @@ def run_host_stack(args, w):
     }))
 
 
+def run_unique_growth(args):
+    """Distinct table rows touched as a function of context length (paper Section 3.2.5: the STEM
+    parameters a sequence activates are |S| d_ff L_uniq, and L_uniq grows sublinearly): one sequence
+    of L positions with the long-context id mix, deduplicated on the GPU, L = 4k ... 128k."""
+    import torch
+    from paper_2601_10639_b200 import binding as B
+    from paper_2601_10639_b200 import runner
+
+    torch.cuda.set_device(0)
+    w = synth.WORKLOADS["1b_long_fwd"]
+    rows = []
+    for L in (4096, 8192, 16384, 32768, 65536, 131072):
+        ids = synth.token_ids(args.seed, L, w.V, w.id_dist)
+        st = runner.LayerState(B.make_shape(L, 8, 8, w.V, B.DTYPE_BF16, B.DTYPE_FP32, 0)).allocate(backward=False)
+        st.ids = torch.from_numpy(ids).cuda()
+        for _ in range(3):
+            st.dedup()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            st.dedup()
+        e1.record()
+        torch.cuda.synchronize()
+        n_u = int(st.bufs["n_unique"].item())
+        assert n_u == len(np.unique(ids)) and st.status() == B.OK
+        rows.append({"L": L, "unique_rows": n_u, "unique_fraction": n_u / L, "dedup_us": 1e3 * e0.elapsed_time(e1) / 20,
+                     "row_bytes_per_layer": n_u * w.d_ff * 2})
+    print(json.dumps({"metric": "distinct table rows touched vs context length", "unit": "rows", "data": "synthetic",
+                      "config": {"workload": "unique_growth", "V": w.V, "d_ff": w.d_ff, "ids": w.id_dist}, "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -314,6 +346,7 @@ def main():
     ap.add_argument("--seed", type=int, default=synth.BASE_SEED)
     ap.add_argument("--tokens", type=int, default=0,
                     help="override the workload's token count (small cases for profiler captures; not a bench line)")
+    ap.add_argument("--unique-growth", action="store_true", help="print distinct rows vs context length and exit")
     ap.add_argument("--grad-bf16", action="store_true", help="host-table workload: bf16 weight and table gradients")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
     args = ap.parse_args()
@@ -323,6 +356,9 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    if args.unique_growth:
+        run_unique_growth(args)
         return
 
     if w.host_tables:
