@@ -26,6 +26,29 @@ __host__ __device__ inline Split make_split(int T) {
   return {n_ctas, epw};
 }
 
+// The kernels of one dedup call are launched with programmatic stream serialisation: each
+// may be scheduled while its predecessor is still draining, waits here for the predecessor's
+// results to be complete and visible, and then lets its own successor be scheduled.  That
+// takes most of the launch gaps out of a chain of six few-microsecond kernels.
+__device__ __forceinline__ void pdl_wait_then_release() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), int grid, int block, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3(static_cast<unsigned>(block));
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ int clamp_id(int key, int V) { return key < 0 ? 0 : (key >= V ? V - 1 : key); }
 
 // Per-warp digit histograms of this CTA's keys, in shared memory.
@@ -53,6 +76,7 @@ __device__ __forceinline__ void warp_histograms(int (*hist)[kRadix], int T, int 
 __global__ void __launch_bounds__(kCtaThreads)
 radix_count_kernel(int T, int V, int epw, int shift, bool first_pass, const int32_t* __restrict__ keys_in,
                    int32_t* __restrict__ cta_hist, int32_t* status) {
+  pdl_wait_then_release();
   __shared__ int hist[kWarps][kRadix];
   warp_histograms(hist, T, V, epw, shift, first_pass, keys_in, status);
   __syncthreads();
@@ -70,6 +94,7 @@ __global__ void __launch_bounds__(kCtaThreads)
 radix_scatter_kernel(int T, int V, int epw, int shift, bool first_pass, const int32_t* __restrict__ keys_in,
                      const int32_t* __restrict__ vals_in, const int32_t* __restrict__ cta_hist,
                      int32_t* __restrict__ keys_out, int32_t* __restrict__ vals_out) {
+  pdl_wait_then_release();
   __shared__ int hist[kWarps][kRadix];
   __shared__ int warp_tot[kRadix / 32];
   warp_histograms(hist, T, V, epw, shift, first_pass, keys_in, nullptr);
@@ -131,6 +156,7 @@ __device__ __forceinline__ bool is_head(const int32_t* __restrict__ sorted_ids, 
 // Heads of runs of equal ids, counted per CTA chunk.
 __global__ void __launch_bounds__(kCtaThreads)
 heads_count_kernel(int T, int per_cta, const int32_t* __restrict__ sorted_ids, int32_t* __restrict__ cta_heads) {
+  pdl_wait_then_release();
   const int begin = blockIdx.x * per_cta, end = min(T, begin + per_cta);
   int local = 0;
   for (int p = begin + threadIdx.x; p < end; p += kCtaThreads) local += is_head(sorted_ids, p) ? 1 : 0;
@@ -150,6 +176,7 @@ heads_write_kernel(int T, int per_cta, const int32_t* __restrict__ sorted_ids, c
                    const int32_t* __restrict__ cta_heads, int32_t* __restrict__ unique_ids,
                    int32_t* __restrict__ n_unique, int32_t* __restrict__ inverse,
                    int32_t* __restrict__ seg_offsets) {
+  pdl_wait_then_release();
   __shared__ int warp_sums[kWarps];
   __shared__ int s_before;
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
@@ -243,19 +270,24 @@ cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, 
     const bool first = pass == 0, last = pass == passes - 1;
     int32_t* kout = keys[pass & 1];
     int32_t* vout = last ? perm : vals[pass & 1];
-    radix_count_kernel<<<sp.n_ctas, kCtaThreads, 0, stream>>>(T, V, sp.epw, pass * 8, first, kin, cta_hist, status);
-    radix_scatter_kernel<<<sp.n_ctas, kCtaThreads, 0, stream>>>(T, V, sp.epw, pass * 8, first, kin, vin, cta_hist,
-                                                               kout, vout);
+    cudaError_t e = launch_chained(radix_count_kernel, sp.n_ctas, kCtaThreads, stream, T, V, sp.epw, pass * 8, first,
+                                   kin, cta_hist, status);
+    if (e != cudaSuccess) return e;
+    e = launch_chained(radix_scatter_kernel, sp.n_ctas, kCtaThreads, stream, T, V, sp.epw, pass * 8, first, kin, vin,
+                       static_cast<const int32_t*>(cta_hist), kout, vout);
+    if (e != cudaSuccess) return e;
     count_launches(2);
     kin = kout;
     vin = vout;
   }
   const int per_cta = sp.epw * kWarps;
-  heads_count_kernel<<<sp.n_ctas, kCtaThreads, 0, stream>>>(T, per_cta, kin, cta_heads);
-  heads_write_kernel<<<sp.n_ctas, kCtaThreads, 0, stream>>>(T, per_cta, kin, perm, cta_heads, unique_ids, n_unique,
-                                                           inverse, seg_offsets);
+  cudaError_t e = launch_chained(heads_count_kernel, sp.n_ctas, kCtaThreads, stream, T, per_cta, kin, cta_heads);
+  if (e != cudaSuccess) return e;
+  e = launch_chained(heads_write_kernel, sp.n_ctas, kCtaThreads, stream, T, per_cta, kin,
+                     static_cast<const int32_t*>(perm), static_cast<const int32_t*>(cta_heads), unique_ids, n_unique,
+                     inverse, seg_offsets);
   count_launches(2);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace stem
