@@ -348,6 +348,8 @@ def main():
                     help="override the workload's token count (small cases for profiler captures; not a bench line)")
     ap.add_argument("--unique-growth", action="store_true", help="print distinct rows vs context length and exit")
     ap.add_argument("--grad-bf16", action="store_true", help="host-table workload: bf16 weight and table gradients")
+    ap.add_argument("--no-profile", action="store_true",
+                    help="do not record per-step events inside the timed region (checks what they cost)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
@@ -417,7 +419,7 @@ def main():
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = B.stem_launch_count()
     with ClockSampler(local) as clocks:
-        B.stem_profile_enable(True)
+        B.stem_profile_enable(not args.no_profile)
         barrier()
         t0 = time.time()
         ev0.record(stream)

@@ -247,6 +247,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (CTAS == 2) ptx::cluster_sync(); else __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above touched only this CTA's own resources, so it may overlap the tail of the
+  // previous kernel in the stream; everything below reads or overwrites global memory.
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
 
   int issued = 0;  // producer: k blocks handed to TMA so far
 
@@ -468,6 +472,8 @@ __global__ void __launch_bounds__(256)
 tail_fixup_kernel(int M, int N, int dp_tiles, int tail, int split, int tiles_m, int tiles_n, int group_m,
                   const float* __restrict__ partial, void* __restrict__ out, int out_fp32) {
   constexpr int TM = BM * CTAS;
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
   const int j = blockIdx.x;
   const TileCoord tc = tile_coord(dp_tiles + j, tiles_m, tiles_n, group_m);
   const int r0 = blockIdx.y * 32;
@@ -564,19 +570,26 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = L::kTotal;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CTAS;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC0, tmC1, M, N, K, 8, dp_tiles, sk_split, ep);
   count_launches(1);
   if (e == cudaSuccess && sk_tail > 0) {
-    tail_fixup_kernel<BN, CTAS><<<dim3(sk_tail, BM * CTAS / 32), 256, 0, stream>>>(
-        M, N, dp_tiles, sk_tail, sk_split, tiles_m, tiles_n, 8, static_cast<const float*>(ep.sk_scratch), ep.out,
-        ep.out_fp32);
+    cudaLaunchConfig_t fcfg = {};
+    fcfg.gridDim = dim3(sk_tail, BM * CTAS / 32);
+    fcfg.blockDim = dim3(256);
+    fcfg.stream = stream;
+    fcfg.attrs = attr + 1;
+    fcfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&fcfg, tail_fixup_kernel<BN, CTAS>, M, N, dp_tiles, sk_tail, sk_split, tiles_m, tiles_n, 8,
+                           static_cast<const float*>(ep.sk_scratch), ep.out, static_cast<int>(ep.out_fp32));
     count_launches(1);
   }
   return e != cudaSuccess ? e : cudaGetLastError();

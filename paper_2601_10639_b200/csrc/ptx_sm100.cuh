@@ -61,6 +61,19 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
   }
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------
+// A kernel launched with programmatic stream serialisation may be scheduled while the kernel
+// before it in the stream is still draining.  grid_dependency_wait() returns once that kernel
+// (and so, by induction, every earlier one that also waits first) is complete and its writes
+// are visible; it must precede the first access to anything an earlier kernel produced or
+// still reads.  grid_launch_dependents() lets the next such kernel be scheduled.
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- TMA --------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
