@@ -174,6 +174,22 @@ int stem_prefetch_rows(const stem_shape_t* shape, const int32_t* ids, const int3
                        const void* table, void* dev_cache, void* ws, void* stream);
 
 /*
+ * Row prefetch with an on-device hot set (Section 3.2.4, "Prefetching cost": traffic is cut
+ * further by caching the most frequently used embeddings in the memory the removed
+ * up-projection frees; Section 3.4 names an LFU cache).  As stem_prefetch_rows, but a row
+ * whose id has a slot in the hot set is copied from device memory instead of the table:
+ *   dev_cache[r,:] = hot_slot[ids[r]] >= 0 ? hot_rows[hot_slot[ids[r]],:] : table[ids[r],:]
+ * hot_rows: device [K,d_ff] (dtype), copies of table rows; hot_slot: device int32 [V], slot of
+ * each id or -1.  Which rows to keep hot (and replacing them as frequencies drift) is the
+ * caller's policy; the result equals stem_prefetch_rows' whenever hot_rows mirrors the table.
+ * stats: optional device int32[2], incremented by the number of rows served from the hot
+ * set ([0]) and from the table ([1]).
+ */
+int stem_prefetch_rows_hot(const stem_shape_t* shape, const int32_t* ids, const int32_t* n_ids,
+                           const void* table, const void* hot_rows, const int32_t* hot_slot,
+                           void* dev_cache, int32_t* stats, void* ws, void* stream);
+
+/*
  * Gradient write-back for an off-device table (Table 1 notes: the table's gradients are
  * transferred back to CPU for the optimizer update):
  *   host_rows[r,:] = dE_rows[r,:] for r < *n_rows;  host_ids[r] = unique_ids[r];

@@ -28,7 +28,7 @@ FLAG_SINGLE_CTA = 2
 EXPORTS = (
     "stem_version", "stem_status_string", "stem_workspace_bytes", "stem_init_workspace",
     "stem_query_status", "stem_dedup_ids", "stem_ffn_forward", "stem_ffn_backward",
-    "stem_prefetch_rows", "stem_writeback_rows", "stem_writeback_rows_dma", "stem_gemm_bf16", "stem_step_arena_bytes",
+    "stem_prefetch_rows", "stem_prefetch_rows_hot", "stem_writeback_rows", "stem_writeback_rows_dma", "stem_gemm_bf16", "stem_step_arena_bytes",
     "stem_ffn_step_host", "stem_ffn_step_host_flush", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
     "stem_dedup_ids_static", "stem_dedup_static_max_tokens",
 )
@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
             "stem_ffn_forward": [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
             "stem_ffn_backward": [shp] + [vp] * 17 + [sz, vp],
             "stem_prefetch_rows": [shp, vp, vp, vp, vp, vp, vp],
+            "stem_prefetch_rows_hot": [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp],
             "stem_writeback_rows": [shp, vp, vp, vp, vp, vp, vp, vp],
             "stem_writeback_rows_dma": [shp, vp, vp, i32, vp, vp, vp],
             "stem_gemm_bf16": [i32, i32, i32, vp, i32, vp, i32, vp, i32, i32, vp, vp],
@@ -164,6 +165,11 @@ def stem_ffn_backward(shape, dy, x, ids, W_gate, E, W_down, G_save, H_save, perm
 def stem_prefetch_rows(shape, ids, n_ids, table, dev_cache, ws, stream=None) -> None:
     _check(lib().stem_prefetch_rows(ctypes.byref(shape), _p(ids), _p(n_ids), _p(table), _p(dev_cache), _p(ws),
                                     _stream(stream)), "stem_prefetch_rows")
+
+
+def stem_prefetch_rows_hot(shape, ids, n_ids, table, hot_rows, hot_slot, dev_cache, stats, ws, stream=None) -> None:
+    _check(lib().stem_prefetch_rows_hot(ctypes.byref(shape), _p(ids), _p(n_ids), _p(table), _p(hot_rows), _p(hot_slot),
+                                        _p(dev_cache), _p(stats), _p(ws), _stream(stream)), "stem_prefetch_rows_hot")
 
 
 def stem_writeback_rows(shape, dE_rows, unique_ids, n_rows, host_rows, host_ids, host_n, stream=None) -> None:

@@ -333,8 +333,28 @@ int stem_prefetch_rows(const stem_shape_t* shape, const int32_t* ids, const int3
   const int max_rows = shape->T < shape->V ? shape->T : shape->V;
   const size_t row_bytes = static_cast<size_t>(shape->d_ff) * elem_bytes(shape->dtype);
   ProfScope prof("prefetch_rows", static_cast<cudaStream_t>(stream));
-  cudaError_t e = launch_gather_rows(max_rows, shape->V, row_bytes, ids, n_ids, src, on_host, dev_cache,
-                                     ws ? status_of(ws) : nullptr, static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_gather_rows(max_rows, shape->V, row_bytes, ids, n_ids, src, on_host, nullptr, nullptr,
+                                     dev_cache, ws ? status_of(ws) : nullptr, nullptr,
+                                     static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
+int stem_prefetch_rows_hot(const stem_shape_t* shape, const int32_t* ids, const int32_t* n_ids, const void* table,
+                           const void* hot_rows, const int32_t* hot_slot, void* dev_cache, int32_t* stats, void* ws,
+                           void* stream) {
+  if (int rc = check_shape(shape)) return rc;
+  if (shape->T == 0) return STEM_OK;
+  if (!ids || !n_ids || !table || !dev_cache || !hot_rows || !hot_slot || !aligned16(table) || !aligned16(dev_cache) ||
+      !aligned16(hot_rows))
+    return STEM_ERR_INVALID_ARG;
+  const void* src = nullptr;
+  bool on_host = false;
+  if (int rc = pinned_or_device(table, &src, &on_host)) return rc;
+  const int max_rows = shape->T < shape->V ? shape->T : shape->V;
+  const size_t row_bytes = static_cast<size_t>(shape->d_ff) * elem_bytes(shape->dtype);
+  ProfScope prof("prefetch_rows", static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_gather_rows(max_rows, shape->V, row_bytes, ids, n_ids, src, on_host, hot_rows, hot_slot,
+                                     dev_cache, ws ? status_of(ws) : nullptr, stats, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
 }
 

@@ -21,7 +21,8 @@ constexpr int kHostLinkThreads = 128;
 __global__ void __launch_bounds__(kThreads)
 gather_rows_kernel(int V, int vec_per_row, const int32_t* __restrict__ ids,
                    const int32_t* __restrict__ n_ids, const uint4* __restrict__ table,
-                   uint4* __restrict__ dst, int32_t* status) {
+                   const uint4* __restrict__ hot_rows, const int32_t* __restrict__ hot_slot,
+                   uint4* __restrict__ dst, int32_t* status, int32_t* stats) {
   const int n = *n_ids;
   // a CTA handles `rows_per_cta` rows per step so short rows still fill the block
   const int lanes_per_row = min(vec_per_row, static_cast<int>(blockDim.x));
@@ -34,7 +35,11 @@ gather_rows_kernel(int V, int vec_per_row, const int32_t* __restrict__ ids,
       if (lane == 0) report_error(status, STEM_ERR_ID_RANGE, r);
       id = id < 0 ? 0 : V - 1;
     }
-    const uint4* src = table + static_cast<size_t>(id) * vec_per_row;
+    // a row held in the on-device hot set is copied from there instead of crossing the host link
+    const int slot = hot_slot != nullptr ? hot_slot[id] : -1;
+    const uint4* src = slot >= 0 ? hot_rows + static_cast<size_t>(slot) * vec_per_row
+                                 : table + static_cast<size_t>(id) * vec_per_row;
+    if (stats != nullptr && lane == 0) atomicAdd(stats + (slot >= 0 ? 0 : 1), 1);
     uint4* out = dst + static_cast<size_t>(r) * vec_per_row;
     int c = lane;
     for (; c + 7 * lanes_per_row < vec_per_row; c += 8 * lanes_per_row) {
@@ -85,8 +90,9 @@ cudaError_t prefer_max_shared(Kernel kernel) {
 }  // namespace
 
 cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int32_t* ids,
-                               const int32_t* n_ids, const void* table, bool table_on_host, void* dst,
-                               int32_t* status, cudaStream_t stream) {
+                               const int32_t* n_ids, const void* table, bool table_on_host,
+                               const void* hot_rows, const int32_t* hot_slot, void* dst, int32_t* status,
+                               int32_t* stats, cudaStream_t stream) {
   if (max_rows <= 0) return cudaSuccess;
   const int vec = static_cast<int>(row_bytes / 16);
   const int threads = table_on_host ? kHostLinkThreads : kThreads;
@@ -98,7 +104,8 @@ cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int3
   static const cudaError_t configured = prefer_max_shared(gather_rows_kernel);
   if (configured != cudaSuccess) return configured;
   gather_rows_kernel<<<blocks, threads, 0, stream>>>(V, vec, ids, n_ids, static_cast<const uint4*>(table),
-                                                     static_cast<uint4*>(dst), status);
+                                                    static_cast<const uint4*>(hot_rows), hot_slot,
+                                                    static_cast<uint4*>(dst), status, stats);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -89,8 +89,9 @@ cudaError_t launch_segreduce(int T, int F, int in_dtype, int out_dtype, const vo
 // table_on_host: the table is page-locked host memory read over the host link; the launch
 // is then kept small enough to share the SMs with a running contraction kernel.
 cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int32_t* ids,
-                               const int32_t* n_ids, const void* table, bool table_on_host, void* dst,
-                               int32_t* status, cudaStream_t stream);
+                               const int32_t* n_ids, const void* table, bool table_on_host,
+                               const void* hot_rows, const int32_t* hot_slot, void* dst, int32_t* status,
+                               int32_t* stats, cudaStream_t stream);
 cudaError_t launch_writeback_rows(int max_rows, size_t row_bytes, const void* rows,
                                   const int32_t* unique_ids, const int32_t* n_rows, void* host_rows,
                                   int32_t* host_ids, int32_t* host_n, cudaStream_t stream);

@@ -233,3 +233,88 @@ class HostTableStack:
             for k in self.slots:
                 if k["used"]:
                     self.main.wait_event(k["written"])
+
+
+def build_hot_set(host_table: torch.Tensor, hot_ids: torch.Tensor, device="cuda"):
+    """Device copies of the rows `hot_ids` of a host table and the id -> slot map for
+    stem_prefetch_rows_hot (set-up, outside the hot path)."""
+    V = host_table.shape[0]
+    hot_ids = hot_ids.to(torch.int64).cpu()
+    hot_rows = host_table[hot_ids].to(device)
+    hot_slot = torch.full((V,), -1, dtype=torch.int32)
+    hot_slot[hot_ids] = torch.arange(hot_ids.numel(), dtype=torch.int32)
+    return hot_rows, hot_slot.to(device)
+
+
+class HostTablePrefill:
+    """Forward-only pass (prefill) through a stack of STEM layers whose tables live in host memory
+    (paper Section 3.4, inference: tables offloaded to CPU, token ids deduplicated, rows prefetched
+    asynchronously with layer computation; Section 3.2.4: frequent rows cached on the device).
+
+    All layers of a model see the same token ids, so they are deduplicated once; layer l+1's rows
+    are gathered on a side stream while layer l computes (two row caches).  With `hot` (one
+    (hot_rows, hot_slot) pair per layer) rows in the on-device hot set do not cross the host link.
+    ``resident=True`` reads device-resident tables directly: the reference for exposed copy time.
+    """
+
+    def __init__(self, shape: B.StemShape, layers: int, tables, W_gate, W_down, resident: bool, hot=None,
+                 device="cuda"):
+        self.shape, self.layers, self.tables, self.resident, self.hot = shape, layers, tables, resident, hot
+        self.W_gate, self.W_down = W_gate, W_down
+        s = shape
+        T, d, F = s.T, s.d_model, s.d_ff
+        dt = torch_dtype(s.dtype)
+        R = max(min(T, s.V), 1)
+        self.cache_shape = B.make_shape(T, d, F, R, s.dtype, s.grad_dtype, s.flags)
+        self.main, self.fetch = torch.cuda.current_stream(), torch.cuda.Stream()
+        self.ws = torch.empty(max(B.stem_workspace_bytes(s), 256), dtype=torch.uint8, device=device)
+        B.stem_init_workspace(self.ws)
+        self.y = torch.empty(T, d, dtype=dt, device=device)
+        self.unique_ids = torch.empty(R, dtype=torch.int32, device=device)
+        self.n_unique = torch.zeros(1, dtype=torch.int32, device=device)
+        self.inverse = torch.empty(T, dtype=torch.int32, device=device)
+        self.perm = torch.empty(T, dtype=torch.int32, device=device)
+        self.seg_offsets = torch.empty(R + 1, dtype=torch.int32, device=device)
+        self.stats = torch.zeros(2, dtype=torch.int32, device=device)
+        self.caches = [] if resident else [torch.empty(R, F, dtype=dt, device=device) for _ in range(2)]
+        self.fetched = [torch.cuda.Event() for _ in range(2)]
+        self.fwd_done = [torch.cuda.Event() for _ in range(2)]
+        self.deduped = torch.cuda.Event()
+        self.used = [False, False]
+
+    def _fetch(self, l: int):
+        k = l & 1
+        if self.used[k]:
+            self.fetch.wait_event(self.fwd_done[k])        # the cache is still being read by layer l-2
+        if self.hot is not None:
+            hot_rows, hot_slot = self.hot[l]
+            B.stem_prefetch_rows_hot(self.shape, self.unique_ids, self.n_unique, self.tables[l], hot_rows, hot_slot,
+                                     self.caches[k], self.stats, self.ws, self.fetch)
+        else:
+            B.stem_prefetch_rows(self.shape, self.unique_ids, self.n_unique, self.tables[l], self.caches[k], self.ws,
+                                 self.fetch)
+        self.fetched[k].record(self.fetch)
+
+    def run(self, xs, ids, on_layer=None):
+        """xs: one [T, d_model] input per layer (the layers are independent here); ids: [T]."""
+        B.stem_dedup_ids(self.shape, ids, self.unique_ids, self.n_unique, self.inverse, self.perm, self.seg_offsets,
+                         self.ws, self.main)
+        if not self.resident:
+            self.deduped.record(self.main)
+            self.fetch.wait_event(self.deduped)
+            self._fetch(0)
+        for l in range(self.layers):
+            k = l & 1
+            if self.resident:
+                B.stem_ffn_forward(self.shape, xs[l], ids, self.W_gate, self.tables[l], self.W_down, self.y, None, None,
+                                   self.ws, self.main)
+            else:
+                if l + 1 < self.layers:
+                    self._fetch(l + 1)
+                self.main.wait_event(self.fetched[k])
+                B.stem_ffn_forward(self.cache_shape, xs[l], self.inverse, self.W_gate, self.caches[k], self.W_down,
+                                   self.y, None, None, self.ws, self.main)
+                self.fwd_done[k].record(self.main)
+                self.used[k] = True
+            if on_layer is not None:
+                on_layer(l)

@@ -371,6 +371,63 @@ def test_host_table_stack_matches_resident_layers():
         assert torch.equal(k["host_rows"][:n], refs[l]["dE"]) and torch.equal(k["host_ids"][:n], refs[l]["uid"])
 
 
+def test_prefetch_with_hot_set_and_prefill_stack():
+    """Rows served from an on-device hot set or from the host table give the same row cache as the
+    plain prefetch (and the checker's row copy); a forward-only stack with shared ids, prefetch on a
+    side stream and per-layer hot sets reproduces every layer's y."""
+    w = synth.Workload("t", 900, 256, 512, 2000, "bf16", "mix")
+    L = 4
+    shape = B.make_shape(w.T, w.d_model, w.d_ff, w.V, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    inps = [synth.make_inputs(w, seed=110, layer=l) for l in range(L)]
+    ids_np = inps[0]["ids"]
+    ids = runner.to_device(ids_np, B.DTYPE_BF16)
+    W_gate = runner.to_device(inps[0]["W_gate"], B.DTYPE_BF16)
+    W_down = runner.to_device(inps[0]["W_down"], B.DTYPE_BF16)
+    xs = [runner.to_device(i["x"], B.DTYPE_BF16) for i in inps]
+    dev_tables = [runner.to_device(i["E"], B.DTYPE_BF16) for i in inps]
+    host_tables = [t.cpu().pin_memory() for t in dev_tables]
+    hot_ids = torch.arange(0, 300)                                  # the most frequent ids of the Zipf part
+    hot = [runner.build_hot_set(t, hot_ids) for t in host_tables]
+    dd = O.dedup(ids_np)
+    n_u = dd["n_unique"]
+    # the gather alone
+    st = runner.LayerState(shape).allocate(backward=False)
+    st.ids = ids
+    st.dedup()
+    cache = torch.zeros(min(w.T, w.V), w.d_ff, dtype=torch.bfloat16, device="cuda")
+    stats = torch.zeros(2, dtype=torch.int32, device="cuda")
+    B.stem_prefetch_rows_hot(shape, st.bufs["unique_ids"], st.bufs["n_unique"], host_tables[1], hot[1][0], hot[1][1],
+                             cache, stats, st.bufs["ws"])
+    torch.cuda.synchronize()
+    expect = O.prefetch_rows(dd["unique_ids"], n_u, inps[1]["E"])
+    assert np.array_equal(cache[:n_u].float().cpu().numpy(), expect)
+    assert torch.count_nonzero(cache[n_u:]) == 0
+    n_hot = int((dd["unique_ids"] < 300).sum())
+    assert stats.tolist() == [n_hot, n_u - n_hot] and 0 < n_hot < n_u
+    # the stack
+    refs = []
+    for l in range(L):
+        one = runner.LayerState(shape)
+        one.x, one.ids, one.W_gate, one.W_down, one.E = xs[l], ids, W_gate, W_down, dev_tables[l]
+        one.allocate(backward=False)
+        one.forward(save=False)
+        torch.cuda.synchronize()
+        refs.append(one.bufs["y"].clone())
+    for mode in ("resident", "host", "hot"):
+        stack = runner.HostTablePrefill(shape, L, dev_tables if mode == "resident" else host_tables, W_gate, W_down,
+                                        mode == "resident", hot if mode == "hot" else None)
+        got = []
+        for _ in range(2):                                      # twice: the cache slots are reused
+            got.clear()
+            stack.run(xs, ids, on_layer=lambda l: got.append(stack.y.clone()))
+        torch.cuda.synchronize()
+        assert B.stem_query_status(stack.ws) == B.OK
+        for l in range(L):
+            assert torch.equal(got[l], refs[l]), (mode, l)
+        if mode == "hot":
+            assert stack.stats.tolist() == [2 * L * n_hot, 2 * L * (n_u - n_hot)]
+
+
 def test_step_from_host_buffers_pipelined():
     """Three back-to-back calls with different batches (the two buffer slots are both reused):
     each must return exactly what the device-resident path computes for its batch."""
