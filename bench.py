@@ -302,6 +302,93 @@ def run_host_stack(args, w):
     }))
 
 
+def run_prefill_stack(args, w):
+    """Forward-only pass of one long sequence through a stack of layers with host-resident tables:
+    ids deduplicated once, rows prefetched a layer ahead, with and without an on-device hot set."""
+    import torch
+    from paper_2601_10639_b200 import binding as B
+    from paper_2601_10639_b200 import runner
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    B.lib()
+    dt = torch.bfloat16
+    T, d, F, V, L = (args.tokens or w.T), w.d_model, w.d_ff, w.V, w.layers
+    gen = torch.Generator(device=dev).manual_seed(args.seed)
+    shape = B.make_shape(T, d, F, V, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    W_gate = (torch.randn(F, d, generator=gen, device=dev) * d ** -0.5).to(dt)
+    W_down = (torch.randn(d, F, generator=gen, device=dev) * F ** -0.5).to(dt)
+    xs = [torch.randn(T, d, generator=gen, device=dev).to(dt) for _ in range(L)]
+    ids_np = synth.token_ids(args.seed, T, V, w.id_dist)
+    ids = torch.from_numpy(ids_np).to(dev)
+    dev_tables, host_tables = [], []
+    for l in range(L):
+        E = torch.empty(V, F, device=dev, dtype=dt)
+        for r0 in range(0, V, 4096):
+            r1 = min(V, r0 + 4096)
+            E[r0:r1] = (torch.randn(r1 - r0, F, generator=gen, device=dev) * 0.02).to(dt)
+        dev_tables.append(E)
+        h = torch.empty(V, F, dtype=dt).pin_memory()
+        h.copy_(E)
+        host_tables.append(h)
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+    uniq = np.unique(ids_np)
+    n_u = int(uniq.size)
+    results = {}
+    # hot sets: the K most frequent ids of the token distribution (ids are frequency-ranked, so 0..K-1)
+    modes = [("resident", None), ("host", None)] + [(f"host+hot{K}", K) for K in args.hot_rows]
+    for name, K in modes:
+        hot = None
+        if K:
+            hot = [runner.build_hot_set(t, torch.arange(0, K)) for t in host_tables]
+        stack = runner.HostTablePrefill(shape, L, dev_tables if name == "resident" else host_tables, W_gate, W_down,
+                                        name == "resident", hot)
+        for _ in range(args.warmup):
+            stack.run(xs, ids)
+        torch.cuda.synchronize()
+        stack.stats.zero_()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with ClockSampler(0) as clocks:
+            t0 = time.time()
+            ev0.record(stream)
+            for _ in range(args.steps):
+                stack.run(xs, ids)
+            ev1.record(stream)
+            torch.cuda.synchronize()
+            t1 = time.time()
+        assert B.stem_query_status(stack.ws) == B.OK and int(stack.n_unique.item()) == n_u
+        ms = ev0.elapsed_time(ev1) / args.steps
+        r = {"ms_per_step": ms, "ms_per_layer": ms / L, "clocks": clocks.summary(t0, t1)}
+        if K:
+            hits, misses = stack.stats.tolist()
+            assert hits + misses == args.steps * L * n_u
+            r.update(hot_rows=K, hot_bytes_per_layer=K * F * 2, unique_row_hit_rate=hits / (hits + misses),
+                     token_hit_rate=float((ids_np < K).mean()), rows_over_link_per_layer=misses / (args.steps * L))
+        results[name] = r
+        del stack, hot
+    res_ms = results["resident"]["ms_per_step"]
+    for name, r in results.items():
+        r["exposed_copy_ms_per_layer"] = (r["ms_per_step"] - res_ms) / L
+    best = min((r["ms_per_step"], n) for n, r in results.items() if n != "resident")[1]
+    ms = results[best]["ms_per_step"]
+    peaks = load_peaks()
+    tf = layer_flops(T, d, F, False) * L / (ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": "STEM-FFN forward tokens/sec (prefill through a stack with host-resident tables)",
+        "value": L * T / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": w.name, "layers": L, "T": T, "d_model": d, "d_ff": F, "V": V, "ids": w.id_dist,
+                   "n_unique": n_u, "reported_mode": best, "l2": "working set exceeds L2; no flush"},
+        "clocks": results[best]["clocks"], "tflops_step": tf, "modes": results,
+        "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": tf / peaks["bf16_tflops_sustained"], "traffic": None,
+                     "peak_source": peaks["source"] + " (sustained bf16 GEMM, of measured)",
+                     "kernel": "whole pass (two contractions per layer)"},
+    }))
+
+
 def run_unique_growth(args):
     """Distinct table rows touched as a function of context length (paper Section 3.2.5: the STEM
     parameters a sequence activates are |S| d_ff L_uniq, and L_uniq grows sublinearly): one sequence
@@ -346,6 +433,8 @@ def main():
     ap.add_argument("--seed", type=int, default=synth.BASE_SEED)
     ap.add_argument("--tokens", type=int, default=0,
                     help="override the workload's token count (small cases for profiler captures; not a bench line)")
+    ap.add_argument("--hot-rows", type=int, nargs="*", default=[2048, 8192],
+                    help="prefill workload: sizes of the on-device hot set to try")
     ap.add_argument("--unique-growth", action="store_true", help="print distinct rows vs context length and exit")
     ap.add_argument("--grad-bf16", action="store_true", help="host-table workload: bf16 weight and table gradients")
     ap.add_argument("--no-profile", action="store_true",
@@ -366,7 +455,10 @@ def main():
     if w.host_tables:
         if int(os.environ.get("WORLD_SIZE", "1")) > 1:
             raise SystemExit("the host-table workload is a one-GPU measurement")
-        run_host_stack(args, w)
+        if w.backward:
+            run_host_stack(args, w)
+        else:
+            run_prefill_stack(args, w)
         return
 
     import torch

@@ -168,6 +168,9 @@ WORKLOADS = {
     # long-context forward only, one sequence of 32768 tokens
     "1b_long_fwd": Workload("1b_long_fwd", 32768, 2048, 8192, 32000, "bf16", "mix", backward=False),
     # 16 independent 1B-class layers, tables in pinned host memory
+    # long-context prefill through 16 layers, tables in pinned host memory, optional hot rows on the device
+    "1b_prefill_host_x16": Workload("1b_prefill_host_x16", 32768, 2048, 8192, 32000, "bf16", "mix",
+                                    backward=False, layers=16, host_tables=True),
     "1b_host_x16": Workload("1b_host_x16", 16384, 2048, 8192, 32000, "bf16", "zipf",
                             layers=16, host_tables=True),
 }
