@@ -190,6 +190,31 @@ int stem_prefetch_rows_hot(const stem_shape_t* shape, const int32_t* ids, const 
                            void* dev_cache, int32_t* stats, void* ws, void* stream);
 
 /*
+ * Frequency-ranked ("LFU") maintenance of the hot set used by stem_prefetch_rows_hot, for
+ * decoding with an off-device table (Section 3.4: token ids are Zipfian, so a memory-efficient
+ * LFU cache serves most lookups -- the paper reports more than 80 % hits; Section 3.2.4: the
+ * cache lives in the memory the removed up-projection frees).  State, all caller-owned device
+ * memory, initialised by the caller: freq int32 [V] = 0, hot_slot int32 [V] = -1, hot_ids
+ * int32 [K] = -1 (id held by each slot), hot_rows [K,d_ff].
+ *   stem_lfu_touch    one decode step's lookups: freq[ids[i]] += 1 for i < n; stats (optional
+ *                     device int32[2]) += {lookups the cache serves, lookups it misses}.
+ *   stem_lfu_refresh  afterwards the cache holds exactly the K ids with the largest freq (ties
+ *                     to the smaller id; ids with freq 0 are never cached): ids that dropped
+ *                     out lose their slots, ids that came in take them and their rows are
+ *                     copied from `table` (page-locked host or device memory, [V,d_ff]).  Which
+ *                     slot an id gets is arbitrary.  *n_installed (optional device int32) =
+ *                     rows copied.  lfu_ws: device scratch of stem_lfu_workspace_bytes(V, K).
+ * The paper gives no algorithm for its cache; this is least-frequently-used eviction applied
+ * in batches (call refresh every few steps).
+ */
+int stem_lfu_workspace_bytes(int32_t V, int32_t K, size_t* bytes /*host, out*/);
+int stem_lfu_touch(int32_t n, int32_t V, const int32_t* ids, int32_t* freq, const int32_t* hot_slot,
+                   int32_t* stats, void* stream);
+int stem_lfu_refresh(const stem_shape_t* shape, int32_t K, const int32_t* freq, int32_t* hot_slot,
+                     int32_t* hot_ids, void* hot_rows, const void* table, int32_t* n_installed,
+                     void* lfu_ws, size_t lfu_ws_bytes, void* stream);
+
+/*
  * Gradient write-back for an off-device table (Table 1 notes: the table's gradients are
  * transferred back to CPU for the optimizer update):
  *   host_rows[r,:] = dE_rows[r,:] for r < *n_rows;  host_ids[r] = unique_ids[r];

@@ -141,6 +141,21 @@ def prefetch_rows(unique_ids, n_ids: int, host_E) -> np.ndarray:
     return np.asarray(host_E)[idx].copy()
 
 
+def lfu_hot_set(freq, K: int) -> np.ndarray:
+    """Ids a frequency-ranked cache of K rows holds (Section 3.4 names an LFU cache; no algorithm
+    is given): the K ids with the largest lookup counts, ties to the smaller id, never an id
+    that was not looked up.  Returned ascending."""
+    freq = np.asarray(freq, dtype=np.int64)
+    order = np.lexsort((np.arange(freq.shape[0]), -freq))      # by count descending, then id
+    top = order[:K]
+    return np.sort(top[freq[top] > 0]).astype(np.int32)
+
+
+def lfu_hits(ids, hot_ids) -> int:
+    """Lookups of one decode step that a cache holding `hot_ids` serves."""
+    return int(np.isin(np.asarray(ids), np.asarray(hot_ids)).sum())
+
+
 def ffn_macs_per_token(d: int, d_ff: int, stem: bool) -> int:
     """Multiply-accumulates of one FFN layer per token, forward (Table 1, row "FLOPs", with the
     element-wise term left out as the paper's text does): three d x d_ff products for a dense

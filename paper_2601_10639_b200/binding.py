@@ -28,7 +28,7 @@ FLAG_SINGLE_CTA = 2
 EXPORTS = (
     "stem_version", "stem_status_string", "stem_workspace_bytes", "stem_init_workspace",
     "stem_query_status", "stem_dedup_ids", "stem_ffn_forward", "stem_ffn_backward",
-    "stem_prefetch_rows", "stem_prefetch_rows_hot", "stem_writeback_rows", "stem_writeback_rows_dma", "stem_gemm_bf16", "stem_step_arena_bytes",
+    "stem_prefetch_rows", "stem_prefetch_rows_hot", "stem_lfu_workspace_bytes", "stem_lfu_touch", "stem_lfu_refresh", "stem_writeback_rows", "stem_writeback_rows_dma", "stem_gemm_bf16", "stem_step_arena_bytes",
     "stem_ffn_step_host", "stem_ffn_step_host_flush", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
     "stem_dedup_ids_static", "stem_dedup_static_max_tokens",
 )
@@ -70,6 +70,9 @@ def lib() -> ctypes.CDLL:
             "stem_ffn_backward": [shp] + [vp] * 17 + [sz, vp],
             "stem_prefetch_rows": [shp, vp, vp, vp, vp, vp, vp],
             "stem_prefetch_rows_hot": [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp],
+            "stem_lfu_workspace_bytes": [i32, i32, ctypes.POINTER(sz)],
+            "stem_lfu_touch": [i32, i32, vp, vp, vp, vp, vp],
+            "stem_lfu_refresh": [shp, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp],
             "stem_writeback_rows": [shp, vp, vp, vp, vp, vp, vp, vp],
             "stem_writeback_rows_dma": [shp, vp, vp, i32, vp, vp, vp],
             "stem_gemm_bf16": [i32, i32, i32, vp, i32, vp, i32, vp, i32, i32, vp, vp],
@@ -170,6 +173,22 @@ def stem_prefetch_rows(shape, ids, n_ids, table, dev_cache, ws, stream=None) -> 
 def stem_prefetch_rows_hot(shape, ids, n_ids, table, hot_rows, hot_slot, dev_cache, stats, ws, stream=None) -> None:
     _check(lib().stem_prefetch_rows_hot(ctypes.byref(shape), _p(ids), _p(n_ids), _p(table), _p(hot_rows), _p(hot_slot),
                                         _p(dev_cache), _p(stats), _p(ws), _stream(stream)), "stem_prefetch_rows_hot")
+
+
+def stem_lfu_workspace_bytes(V: int, K: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().stem_lfu_workspace_bytes(V, K, ctypes.byref(out)), "stem_lfu_workspace_bytes")
+    return out.value
+
+
+def stem_lfu_touch(n: int, V: int, ids, freq, hot_slot, stats=None, stream=None) -> None:
+    _check(lib().stem_lfu_touch(n, V, _p(ids), _p(freq), _p(hot_slot), _p(stats), _stream(stream)), "stem_lfu_touch")
+
+
+def stem_lfu_refresh(shape, K: int, freq, hot_slot, hot_ids, hot_rows, table, n_installed, lfu_ws, stream=None) -> None:
+    _check(lib().stem_lfu_refresh(ctypes.byref(shape), K, _p(freq), _p(hot_slot), _p(hot_ids), _p(hot_rows), _p(table),
+                                  _p(n_installed), _p(lfu_ws), lfu_ws.numel() * lfu_ws.element_size(),
+                                  _stream(stream)), "stem_lfu_refresh")
 
 
 def stem_writeback_rows(shape, dE_rows, unique_ids, n_rows, host_rows, host_ids, host_n, stream=None) -> None:

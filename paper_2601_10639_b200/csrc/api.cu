@@ -358,6 +358,39 @@ int stem_prefetch_rows_hot(const stem_shape_t* shape, const int32_t* ids, const 
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
 }
 
+int stem_lfu_workspace_bytes(int32_t V, int32_t K, size_t* bytes) {
+  if (!bytes || V <= 0 || K <= 0 || K > V || V > (1 << 30)) return STEM_ERR_INVALID_ARG;
+  *bytes = lfu_workspace_bytes(V, K);
+  return STEM_OK;
+}
+
+int stem_lfu_touch(int32_t n, int32_t V, const int32_t* ids, int32_t* freq, const int32_t* hot_slot,
+                   int32_t* stats, void* stream) {
+  if (n < 0 || V <= 0) return STEM_ERR_INVALID_ARG;
+  if (n == 0) return STEM_OK;
+  if (!ids || !freq || !hot_slot) return STEM_ERR_INVALID_ARG;
+  ProfScope prof("lfu_touch", static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_lfu_touch(n, V, ids, freq, hot_slot, stats, nullptr, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
+int stem_lfu_refresh(const stem_shape_t* shape, int32_t K, const int32_t* freq, int32_t* hot_slot, int32_t* hot_ids,
+                     void* hot_rows, const void* table, int32_t* n_installed, void* lfu_ws, size_t lfu_ws_bytes,
+                     void* stream) {
+  if (int rc = check_shape(shape)) return rc;
+  if (K <= 0 || K > shape->V || !freq || !hot_slot || !hot_ids || !hot_rows || !table || !lfu_ws ||
+      !aligned16(hot_rows) || !aligned16(table) || !aligned16(lfu_ws))
+    return STEM_ERR_INVALID_ARG;
+  if (lfu_ws_bytes < lfu_workspace_bytes(shape->V, K)) return STEM_ERR_WORKSPACE_TOO_SMALL;
+  const void* src = nullptr;
+  if (int rc = pinned_or_device(table, &src)) return rc;
+  const size_t row_bytes = static_cast<size_t>(shape->d_ff) * elem_bytes(shape->dtype);
+  ProfScope prof("lfu_refresh", static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_lfu_refresh(shape->V, K, row_bytes, freq, hot_slot, hot_ids, hot_rows, src, n_installed, lfu_ws,
+                                     static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
 int stem_writeback_rows(const stem_shape_t* shape, const void* dE_rows, const int32_t* unique_ids,
                         const int32_t* n_rows, void* host_rows, int32_t* host_ids, int32_t* host_n,
                         void* stream) {

@@ -247,6 +247,37 @@ size_t dedup_workspace_bytes(int T, int V) {
   return 4 * align_up(static_cast<size_t>(T) * 4, 256) + static_cast<size_t>(kMaxCtas) * kRadix * 4 + 256;
 }
 
+// Stable LSD radix sort of n keys in [0, V): perm = positions in sorted order; *sorted_keys
+// points at the sorted keys (inside scratch).  scratch: dedup_workspace_bytes(n, V) bytes.
+cudaError_t launch_stable_sort(int n, int V, const int32_t* keys_in, int32_t* perm, void* scratch,
+                               const int32_t** sorted_keys, int32_t* status, cudaStream_t stream) {
+  const Split sp = make_split(n);
+  const size_t tb = align_up(static_cast<size_t>(n) * 4, 256);
+  char* p = static_cast<char*>(scratch);
+  int32_t* keys[2] = {reinterpret_cast<int32_t*>(p), reinterpret_cast<int32_t*>(p + tb)};
+  int32_t* vals[2] = {reinterpret_cast<int32_t*>(p + 2 * tb), reinterpret_cast<int32_t*>(p + 3 * tb)};
+  int32_t* cta_hist = reinterpret_cast<int32_t*>(p + 4 * tb);
+  const int passes = (key_bits(V) + 7) / 8;
+  const int32_t* kin = keys_in;
+  const int32_t* vin = nullptr;
+  for (int pass = 0; pass < passes; ++pass) {
+    const bool first = pass == 0, last = pass == passes - 1;
+    int32_t* kout = keys[pass & 1];
+    int32_t* vout = last ? perm : vals[pass & 1];
+    cudaError_t e = launch_chained(radix_count_kernel, sp.n_ctas, kCtaThreads, stream, n, V, sp.epw, pass * 8, first,
+                                   kin, cta_hist, status);
+    if (e != cudaSuccess) return e;
+    e = launch_chained(radix_scatter_kernel, sp.n_ctas, kCtaThreads, stream, n, V, sp.epw, pass * 8, first, kin, vin,
+                       static_cast<const int32_t*>(cta_hist), kout, vout);
+    if (e != cudaSuccess) return e;
+    count_launches(2);
+    kin = kout;
+    vin = vout;
+  }
+  *sorted_keys = kin;
+  return cudaSuccess;
+}
+
 cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, int32_t* n_unique,
                          int32_t* inverse, int32_t* perm, int32_t* seg_offsets, void* scratch,
                          int32_t* status, cudaStream_t stream) {
@@ -257,29 +288,9 @@ cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, 
   }
   const Split sp = make_split(T);
   const size_t tb = align_up(static_cast<size_t>(T) * 4, 256);
-  char* p = static_cast<char*>(scratch);
-  int32_t* keys[2] = {reinterpret_cast<int32_t*>(p), reinterpret_cast<int32_t*>(p + tb)};
-  int32_t* vals[2] = {reinterpret_cast<int32_t*>(p + 2 * tb), reinterpret_cast<int32_t*>(p + 3 * tb)};
-  int32_t* cta_hist = reinterpret_cast<int32_t*>(p + 4 * tb);
-  int32_t* cta_heads = cta_hist + kMaxCtas * kRadix;
-
-  const int passes = (key_bits(V) + 7) / 8;
-  const int32_t* kin = ids;
-  const int32_t* vin = nullptr;
-  for (int pass = 0; pass < passes; ++pass) {
-    const bool first = pass == 0, last = pass == passes - 1;
-    int32_t* kout = keys[pass & 1];
-    int32_t* vout = last ? perm : vals[pass & 1];
-    cudaError_t e = launch_chained(radix_count_kernel, sp.n_ctas, kCtaThreads, stream, T, V, sp.epw, pass * 8, first,
-                                   kin, cta_hist, status);
-    if (e != cudaSuccess) return e;
-    e = launch_chained(radix_scatter_kernel, sp.n_ctas, kCtaThreads, stream, T, V, sp.epw, pass * 8, first, kin, vin,
-                       static_cast<const int32_t*>(cta_hist), kout, vout);
-    if (e != cudaSuccess) return e;
-    count_launches(2);
-    kin = kout;
-    vin = vout;
-  }
+  int32_t* cta_heads = reinterpret_cast<int32_t*>(static_cast<char*>(scratch) + 4 * tb) + kMaxCtas * kRadix;
+  const int32_t* kin = nullptr;
+  if (cudaError_t e = launch_stable_sort(T, V, ids, perm, scratch, &kin, status, stream)) return e;
   const int per_cta = sp.epw * kWarps;
   cudaError_t e = launch_chained(heads_count_kernel, sp.n_ctas, kCtaThreads, stream, T, per_cta, kin, cta_heads);
   if (e != cudaSuccess) return e;

@@ -78,6 +78,11 @@ cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, 
                          int32_t* inverse, int32_t* perm, int32_t* seg_offsets, void* scratch,
                          int32_t* status, cudaStream_t stream);
 
+// Stable radix sort of n keys in [0, V) (the sort inside launch_dedup): perm = positions in
+// sorted order, *sorted_keys = the sorted keys (inside scratch, dedup_workspace_bytes(n, V)).
+cudaError_t launch_stable_sort(int n, int V, const int32_t* keys_in, int32_t* perm, void* scratch,
+                               const int32_t** sorted_keys, int32_t* status, cudaStream_t stream);
+
 // ---- table-gradient reduce --------------------------------------------------------------
 size_t segreduce_workspace_bytes(int T, int F);
 cudaError_t launch_segreduce(int T, int F, int in_dtype, int out_dtype, const void* dU,
@@ -95,6 +100,14 @@ cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int3
 cudaError_t launch_writeback_rows(int max_rows, size_t row_bytes, const void* rows,
                                   const int32_t* unique_ids, const int32_t* n_rows, void* host_rows,
                                   int32_t* host_ids, int32_t* host_n, cudaStream_t stream);
+
+// ---- frequency-ranked row cache ------------------------------------------------------------
+size_t lfu_workspace_bytes(int V, int K);
+cudaError_t launch_lfu_touch(int n, int V, const int32_t* ids, int32_t* freq, const int32_t* hot_slot,
+                             int32_t* stats, int32_t* status, cudaStream_t stream);
+cudaError_t launch_lfu_refresh(int V, int K, size_t row_bytes, const int32_t* freq, int32_t* hot_slot,
+                               int32_t* hot_ids, void* hot_rows, const void* table, int32_t* n_installed,
+                               void* scratch, cudaStream_t stream);
 
 int device_sm_count();
 void count_launches(int n);  // bookkeeping for stem_launch_count()

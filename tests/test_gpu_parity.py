@@ -428,6 +428,61 @@ def test_prefetch_with_hot_set_and_prefill_stack():
             assert stack.stats.tolist() == [2 * L * n_hot, 2 * L * (n_u - n_hot)]
 
 
+def test_lfu_cache_tracks_the_most_frequent_ids():
+    """Decode steps of Zipfian ids: after every refresh the cache holds exactly the checker's top-K
+    set, every cached row equals its table row, slots are consistent, and the hit counters equal
+    the checker's; a prefetch through the cache returns the plain prefetch's rows."""
+    V, F, K, Bsz = 3000, 512, 64, 97
+    shape = B.make_shape(Bsz, 64, F, V, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    table = torch.from_numpy(synth.round_bf16(synth.normal(5, synth.TAG_E, (V, F), 0.02))).bfloat16().pin_memory()
+    freq = torch.zeros(V, dtype=torch.int32, device="cuda")
+    hot_slot = torch.full((V,), -1, dtype=torch.int32, device="cuda")
+    hot_ids = torch.full((K,), -1, dtype=torch.int32, device="cuda")
+    hot_rows = torch.zeros(K, F, dtype=torch.bfloat16, device="cuda")
+    stats = torch.zeros(2, dtype=torch.int32, device="cuda")
+    n_inst = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lws = torch.empty(B.stem_lfu_workspace_bytes(V, K), dtype=torch.uint8, device="cuda")
+    freq_ref = np.zeros(V, dtype=np.int64)
+    hot_ref = np.array([], dtype=np.int32)
+    hits_ref = 0
+    for step in range(40):
+        ids_np = synth.token_ids(200 + step, Bsz, V, "zipf")
+        ids = torch.from_numpy(ids_np).cuda()
+        B.stem_lfu_touch(Bsz, V, ids, freq, hot_slot, stats)
+        hits_ref += O.lfu_hits(ids_np, hot_ref)
+        np.add.at(freq_ref, ids_np, 1)
+        if step % 4 == 3:
+            B.stem_lfu_refresh(shape, K, freq, hot_slot, hot_ids, hot_rows, table, n_inst, lws)
+            torch.cuda.synchronize()
+            new_ref = O.lfu_hot_set(freq_ref, K)
+            held = hot_ids.cpu().numpy()
+            assert np.array_equal(np.sort(held[held >= 0]), new_ref), step
+            assert int(n_inst.item()) == len(set(new_ref.tolist()) - set(hot_ref.tolist())), step
+            slots = hot_slot.cpu().numpy()
+            assert np.array_equal(np.flatnonzero(slots >= 0), new_ref)
+            for s_, id_ in enumerate(held):
+                if id_ >= 0:
+                    assert slots[id_] == s_
+            rows = hot_rows.cpu()
+            sel = held >= 0
+            assert torch.equal(rows[torch.from_numpy(sel)], table[torch.from_numpy(held[sel]).long()])
+            hot_ref = new_ref
+    torch.cuda.synchronize()
+    assert np.array_equal(freq.cpu().numpy(), freq_ref)
+    assert stats.tolist() == [hits_ref, 40 * Bsz - hits_ref] and hits_ref > 0
+    # prefetch through the cache
+    st = runner.LayerState(shape).allocate(backward=False)
+    st.ids = ids
+    st.dedup()
+    cache = torch.zeros(Bsz, F, dtype=torch.bfloat16, device="cuda")
+    B.stem_prefetch_rows_hot(shape, st.bufs["unique_ids"], st.bufs["n_unique"], table, hot_rows, hot_slot, cache, None,
+                             st.bufs["ws"])
+    torch.cuda.synchronize()
+    dd = O.dedup(ids_np)
+    assert np.array_equal(cache[:dd["n_unique"]].float().numpy(force=True),
+                          O.prefetch_rows(dd["unique_ids"], dd["n_unique"], table.float().numpy()))
+
+
 def test_step_from_host_buffers_pipelined():
     """Three back-to-back calls with different batches (the two buffer slots are both reused):
     each must return exactly what the device-resident path computes for its batch."""

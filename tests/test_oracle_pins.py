@@ -311,3 +311,26 @@ def test_flop_accounting_of_the_benchmark():
     # with all-ones operands every entry of G is the length of its dot product
     assert im["G"].shape == (T, F) and float(im["G"][0, 0]) == d
     assert im["G"].size * d + T * d * F == macs
+
+
+def test_lfu_hot_set_against_brute_force():
+    rng = np.random.default_rng(3)
+    for V, K in ((50, 7), (20, 20), (9, 3)):
+        freq = rng.integers(0, 4, size=V)                       # many ties, some never-seen ids
+        got = O.lfu_hot_set(freq, K)
+        # brute force: repeatedly take the most frequent remaining id (smallest id among equals)
+        left, picked = dict(enumerate(freq.tolist())), []
+        while len(picked) < K and left:
+            best = max(left.values())
+            if best == 0:
+                break
+            i = min(i for i, f in left.items() if f == best)
+            picked.append(i)
+            del left[i]
+        assert got.tolist() == sorted(picked)
+        # nothing outside the set is looked up more often than something inside it
+        if len(picked):
+            inside_min = min(freq[i] for i in picked)
+            assert all(freq[i] <= inside_min for i in range(V) if i not in picked)
+    ids = np.array([1, 1, 5, 7, 7, 7, 2])
+    assert O.lfu_hits(ids, [7, 1]) == 5 and O.lfu_hits(ids, []) == 0
