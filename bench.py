@@ -389,6 +389,110 @@ def run_prefill_stack(args, w):
     }))
 
 
+def run_decode(args, w):
+    """Decode steps with the table in host memory and a frequency-ranked row cache on the device
+    (paper Section 3.4; Table 1, decoding: communication B_uniq * d_ff per step).  A step = count
+    the lookups, deduplicate the step's ids, gather their rows (cache or host link), forward."""
+    import torch
+    from paper_2601_10639_b200 import binding as B
+    from paper_2601_10639_b200 import runner
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    B.lib()
+    dt = torch.bfloat16
+    Bt, d, F, V = (args.tokens or w.T), w.d_model, w.d_ff, w.V
+    steps, refresh_every = max(args.steps, 400), 20
+    gen = torch.Generator(device=dev).manual_seed(args.seed)
+    shape = B.make_shape(Bt, d, F, V, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    cshape = B.make_shape(Bt, d, F, min(Bt, V), B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    W_gate = (torch.randn(F, d, generator=gen, device=dev) * d ** -0.5).to(dt)
+    W_down = (torch.randn(d, F, generator=gen, device=dev) * F ** -0.5).to(dt)
+    x = torch.randn(Bt, d, generator=gen, device=dev).to(dt)
+    E = torch.empty(V, F, device=dev, dtype=dt)
+    for r0 in range(0, V, 4096):
+        r1 = min(V, r0 + 4096)
+        E[r0:r1] = (torch.randn(r1 - r0, F, generator=gen, device=dev) * 0.02).to(dt)
+    table = torch.empty(V, F, dtype=dt).pin_memory()
+    table.copy_(E)
+    del E
+    all_ids = torch.from_numpy(synth.token_ids(args.seed, steps * Bt, V, w.id_dist)).to(dev)   # every step's ids
+    st = runner.LayerState(shape, device=dev).allocate(backward=False)
+    st.x, st.W_gate, st.W_down = x, W_gate, W_down
+    b = st.bufs
+    cache = torch.empty(min(Bt, V), F, dtype=dt, device=dev)
+    stream = torch.cuda.current_stream()
+    out = {}
+    for K in args.hot_rows:
+        freq = torch.zeros(V, dtype=torch.int32, device=dev)
+        hot_slot = torch.full((V,), -1, dtype=torch.int32, device=dev)
+        hot_ids = torch.full((K,), -1, dtype=torch.int32, device=dev)
+        hot_rows = torch.zeros(K, F, dtype=dt, device=dev)
+        stats, rows = torch.zeros(2, dtype=torch.int32, device=dev), torch.zeros(2, dtype=torch.int32, device=dev)
+        n_inst = torch.zeros(1, dtype=torch.int32, device=dev)
+        lws = torch.empty(B.stem_lfu_workspace_bytes(V, K), dtype=torch.uint8, device=dev)
+
+        def step(i):
+            ids = all_ids[i * Bt:(i + 1) * Bt]
+            B.stem_lfu_touch(Bt, V, ids, freq, hot_slot, stats)
+            B.stem_dedup_ids(shape, ids, b["unique_ids"], b["n_unique"], b["inverse"], b["perm"], b["seg_offsets"], b["ws"])
+            B.stem_prefetch_rows_hot(shape, b["unique_ids"], b["n_unique"], table, hot_rows, hot_slot, cache, rows, b["ws"])
+            B.stem_ffn_forward(cshape, x, b["inverse"], W_gate, cache, W_down, b["y"], None, None, b["ws"])
+            if i % refresh_every == refresh_every - 1:
+                B.stem_lfu_refresh(shape, K, freq, hot_slot, hot_ids, hot_rows, table, n_inst, lws)
+
+        half = steps // 2
+        for i in range(half):                       # warm the counters and the cache
+            step(i)
+        torch.cuda.synchronize()
+        stats.zero_(); rows.zero_()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for i in range(half, steps):
+            step(i)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        assert st.status() == B.OK
+        hits, misses = stats.tolist()
+        rhit, rmiss = rows.tolist()
+        n = steps - half
+        out[f"hot{K}"] = {"hot_rows": K, "hot_bytes": K * F * 2, "token_hit_rate": hits / (hits + misses),
+                          "unique_row_hit_rate": rhit / (rhit + rmiss), "unique_rows_per_step": (rhit + rmiss) / n,
+                          "rows_over_link_per_step": rmiss / n, "link_bytes_per_step": rmiss / n * F * 2,
+                          "ms_per_step": ev0.elapsed_time(ev1) / n, "refresh_every_steps": refresh_every}
+    # the same step with the table on the device (no cache, no link): the compute floor of this path
+    dev_table = table.to(dev)
+    def resident_step(i):
+        ids = all_ids[i * Bt:(i + 1) * Bt]
+        B.stem_ffn_forward(shape, x, ids, W_gate, dev_table, W_down, b["y"], None, None, b["ws"])
+    for i in range(20):
+        resident_step(i)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for i in range(200):
+        resident_step(i)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    res_ms = ev0.elapsed_time(ev1) / 200
+    best = min(out.values(), key=lambda r: r["ms_per_step"])
+    peaks = load_peaks()
+    wbytes = 2 * d * F * 2
+    print(json.dumps({
+        "metric": "STEM-FFN decode steps: tokens/sec of one layer with a host-resident table and an LFU row cache",
+        "value": Bt / (best["ms_per_step"] * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": steps - steps // 2,
+        "warmup": steps // 2, "ms_per_step": best["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "tokens_per_step": Bt, "d_model": d, "d_ff": F, "V": V, "ids": w.id_dist,
+                   "paper_hit_rate": "> 80 % (Section 3.4, hardware and cache size not stated)"},
+        "modes": out, "device_table_forward_ms": res_ms,
+        "roofline": {"bound": "hbm", "achieved": wbytes / (res_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": wbytes / (res_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                     "kernel": "forward with a device table (both weight matrices read once per step: 2 d d_ff elements, Table 1)",
+                     "peak_source": peaks["source"] + " (copy bandwidth, of measured)"},
+    }))
+
+
 def run_unique_growth(args):
     """Distinct table rows touched as a function of context length (paper Section 3.2.5: the STEM
     parameters a sequence activates are |S| d_ff L_uniq, and L_uniq grows sublinearly): one sequence
@@ -455,7 +559,9 @@ def main():
     if w.host_tables:
         if int(os.environ.get("WORLD_SIZE", "1")) > 1:
             raise SystemExit("the host-table workload is a one-GPU measurement")
-        if w.backward:
+        if w.note == "decode":
+            run_decode(args, w)
+        elif w.backward:
             run_host_stack(args, w)
         else:
             run_prefill_stack(args, w)
