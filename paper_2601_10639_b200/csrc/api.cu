@@ -250,6 +250,8 @@ int stem_ffn_forward(const stem_shape_t* shape, const void* x, const int32_t* id
   if (e != cudaSuccess) return cuda_fail(e);
   EpiParams down;
   down.out = y; down.out_fp32 = shape->dtype == STEM_DTYPE_FP32; down.status = status_of(ws);
+  // few row tiles and a long contraction (decode steps): the tiles may be cut along k
+  down.sk_scratch = static_cast<char*>(ws) + w.sk_off; down.sk_bytes = w.sk_bytes;
   {
     ProfScope prof("down_gemm", st);
     e = gemm(shape, T, d, F, H, false, W_down, false, kEpiStore, down, st);              // y = H W_down^T
@@ -315,6 +317,7 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
   }
   if (dx) {  // dx = dG W_gate (contraction over d_ff; W_gate is [F, d]: d contiguous)
     EpiParams p; p.out = dx; p.out_fp32 = shape->dtype == STEM_DTYPE_FP32; p.status = status_of(ws);
+    p.sk_scratch = base + w.sk_off; p.sk_bytes = w.sk_bytes;
     ProfScope prof("dx_gemm", st);
     e = gemm(shape, T, d, F, dG, false, W_gate, true, kEpiStore, p, st);
     if (e != cudaSuccess) return cuda_fail(e);

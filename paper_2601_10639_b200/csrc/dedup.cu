@@ -1,7 +1,8 @@
 // Token-id deduplication: a stable LSD radix sort of (id, position) pairs, 8 bits per
 // pass (a count kernel and a scatter kernel per pass), followed by two kernels that mark
 // the head of every run of equal ids and emit the distinct ids, the run offsets and each
-// position's slot.  Integer-only: every output has exactly one correct value.
+// position's slot.  Batches of up to 1024 positions take a one-launch path (rank sort in
+// shared memory).  Integer-only: every output has exactly one correct value.
 #include <mutex>
 
 #include "stem_internal.h"
@@ -227,6 +228,72 @@ heads_write_kernel(int T, int per_cta, const int32_t* __restrict__ sorted_ids, c
   }
 }
 
+// A batch of at most kCtaThreads positions (decode steps) in one launch by one CTA: every
+// thread ranks its own (id, position) pair against all others in shared memory, which is the
+// stable sort; run heads and slots follow from one block-wide scan.  Same outputs as the
+// radix path, without its six launch latencies.
+__global__ void __launch_bounds__(kCtaThreads)
+dedup_small_kernel(int T, int V, const int32_t* __restrict__ ids, int32_t* __restrict__ unique_ids,
+                   int32_t* __restrict__ n_unique, int32_t* __restrict__ inverse, int32_t* __restrict__ perm,
+                   int32_t* __restrict__ seg_offsets, int32_t* status) {
+  __shared__ int s_id[kCtaThreads];       // ids by position, then ids in sorted order
+  __shared__ int s_sorted[kCtaThreads];
+  __shared__ int s_perm[kCtaThreads];
+  __shared__ int s_warp[kWarps];
+  const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+  int id = 0x7fffffff;
+  if (t < T) {
+    id = ids[t];
+    if (id < 0 || id >= V) {
+      if (status != nullptr) { report_error(status, STEM_ERR_ID_RANGE, t); atomicAdd(status + 2, 1); }
+      id = clamp_id(id, V);
+    }
+  }
+  s_id[t] = id;
+  __syncthreads();
+  if (t < T) {
+    int rank = 0;
+    for (int j = 0; j < T; ++j) {
+      const int other = s_id[j];
+      rank += (other < id || (other == id && j < t)) ? 1 : 0;
+    }
+    s_sorted[rank] = id;
+    s_perm[rank] = t;
+  }
+  __syncthreads();
+  // thread t now owns sorted position t
+  const bool head = t < T && (t == 0 || s_sorted[t] != s_sorted[t - 1]);
+  int incl = head ? 1 : 0;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) s_warp[w] = incl;
+  __syncthreads();
+  if (w == 0) {
+    int v = s_warp[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, v, o);
+      if (lane >= o) v += u;
+    }
+    s_warp[lane] = v;
+  }
+  __syncthreads();
+  const int slot = incl + (w > 0 ? s_warp[w - 1] : 0) - 1;   // slot of sorted position t
+  if (t < T) {
+    perm[t] = s_perm[t];
+    if (head) { unique_ids[slot] = s_sorted[t]; seg_offsets[slot] = t; }
+    if (inverse) inverse[s_perm[t]] = slot;
+  }
+  if (t == 0) {
+    const int total = s_warp[kWarps - 1];
+    *n_unique = total;
+    seg_offsets[total] = T;
+  }
+}
+
 __global__ void empty_dedup_kernel(int32_t* n_unique, int32_t* seg_offsets) {
   *n_unique = 0;
   seg_offsets[0] = 0;
@@ -283,6 +350,12 @@ cudaError_t launch_dedup(int T, int V, const int32_t* ids, int32_t* unique_ids, 
                          int32_t* status, cudaStream_t stream) {
   if (T <= 0) {
     empty_dedup_kernel<<<1, 1, 0, stream>>>(n_unique, seg_offsets);
+    count_launches(1);
+    return cudaGetLastError();
+  }
+  if (T <= kCtaThreads) {
+    dedup_small_kernel<<<1, kCtaThreads, 0, stream>>>(T, V, ids, unique_ids, n_unique, inverse, perm, seg_offsets,
+                                                    status);
     count_launches(1);
     return cudaGetLastError();
   }

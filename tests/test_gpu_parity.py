@@ -51,7 +51,7 @@ def test_gemm_layouts(flags, a_mn, b_mn, M, N, K):
 @pytest.mark.parametrize("dist,T,V", [
     ("uniform", 256, 4096), ("zipf", 16384, 32000), ("mix", 32768, 32000), ("same", 1000, 77),
     ("distinct", 3000, 5000), ("uniform", 1, 5), ("uniform", 70001, 300), ("zipf", 100000, 1 << 20),
-    ("uniform", 65, 2), ("uniform", 4097, 1),
+    ("uniform", 65, 2), ("uniform", 4097, 1), ("zipf", 1024, 500), ("zipf", 1025, 500), ("same", 1024, 9),
 ])
 def test_dedup_bit_exact(dist, T, V):
     ids = synth.token_ids(5, T, V, dist)
