@@ -161,6 +161,28 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
                       void* stream);
 
 /*
+ * STEM-dagger (Appendix, "Additional Architecture Ablation Study": the variant that keeps the
+ * up-projection and adds the token's table row to its output):
+ *     y_t = W_down ( SiLU(W_gate x_t) (.) (W_up x_t + E[id_t]) )
+ * Forward: U = x W_up^T + E[ids] (the lookup is added in the up GEMM's epilogue), G = x W_gate^T,
+ * H = SiLU(G) (.) U, y = H W_down^T.  W_up [d_ff,d_model] like W_gate.  U_save [T,d_ff] (dtype) is
+ * a required output (the backward pass needs it); G_save, H_save as in stem_ffn_forward.
+ * Backward (chain rule, as for the layer itself): dH = dy W_down; dU = dH (.) SiLU(G);
+ * dG = dH (.) U (.) SiLU'(G); dW_down = dy^T H; dW_gate = dG^T x; dW_up = dU^T x;
+ * dx = dG W_gate + dU W_up; dE_rows[r] = sum of dU[t] over the positions of unique_ids[r].
+ * perm, seg_offsets, n_unique from stem_dedup_ids; any of dx, dW_gate, dW_up, dW_down, dE_rows
+ * may be NULL.  Same workspace as the layer's calls.
+ */
+int stem_dagger_forward(const stem_shape_t* shape, const void* x, const int32_t* ids, const void* W_gate,
+                        const void* W_up, const void* E, const void* W_down, void* y, void* G_save,
+                        void* H_save, void* U_save, void* ws, size_t ws_bytes, void* stream);
+int stem_dagger_backward(const stem_shape_t* shape, const void* dy, const void* x, const void* W_gate,
+                         const void* W_up, const void* W_down, const void* G_save, const void* H_save,
+                         const void* U_save, const int32_t* perm, const int32_t* seg_offsets,
+                         const int32_t* n_unique, void* dx, void* dW_gate, void* dW_up, void* dW_down,
+                         void* dE_rows, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Row prefetch for a table kept off the device (Section 3.4: tables offloaded to CPU
  * memory, rows of the deduplicated ids prefetched asynchronously with layer compute;
  * Figure 1(c)):   dev_cache[r,:] = table[ids[r],:]   for r < *n_ids.

@@ -127,6 +127,41 @@ def backward(dy, x, ids, W_gate, E, W_down):
     }
 
 
+def dagger_forward(x, ids, W_gate, W_up, E, W_down, return_intermediates: bool = False):
+    """STEM-dagger (Appendix, "STEM-dagger"): y_t = W_d ( SiLU(W_g x_t) (.) (W_u x_t + U[t]) )."""
+    x, W_gate, W_up, W_down = _f64(x), _f64(W_gate), _f64(W_up), _f64(W_down)
+    ids = np.asarray(ids, dtype=np.int64)
+    G = x @ W_gate.T
+    A = silu(G)
+    U = x @ W_up.T + _f64(E[ids])       # the up-projection plus the looked-up row
+    H = A * U
+    y = H @ W_down.T
+    if return_intermediates:
+        return y, {"G": G, "A": A, "U": U, "H": H}
+    return y
+
+
+def dagger_backward(dy, x, ids, W_gate, W_up, E, W_down):
+    """Chain rule of `dagger_forward` for L = sum dy * y (the paper gives no formulas)."""
+    dy, x, W_gate, W_up, W_down = _f64(dy), _f64(x), _f64(W_gate), _f64(W_up), _f64(W_down)
+    ids = np.asarray(ids, dtype=np.int64)
+    _, im = dagger_forward(x, ids, W_gate, W_up, E, W_down, return_intermediates=True)
+    G, A, U, H = im["G"], im["A"], im["U"], im["H"]
+    dH = dy @ W_down
+    dW_down = dy.T @ H
+    dU = dH * A                         # reaches both W_up (through W_u x) and the table row
+    dG = dH * U * silu_grad(G)
+    dW_gate = dG.T @ x
+    dW_up = dU.T @ x
+    dx = dG @ W_gate + dU @ W_up
+    unique_ids = np.unique(ids)
+    dE_rows = np.zeros((unique_ids.shape[0], dU.shape[1]), dtype=np.float64)
+    for r, v in enumerate(unique_ids):
+        dE_rows[r] = dU[ids == v].sum(axis=0)
+    return {"dx": dx, "dW_gate": dW_gate, "dW_up": dW_up, "dW_down": dW_down,
+            "unique_ids": unique_ids.astype(np.int32), "dE_rows": dE_rows}
+
+
 def dE_dense(unique_ids, dE_rows, V: int) -> np.ndarray:
     """Scatter the compact table gradient into a [V,F] array (absent ids stay zero)."""
     out = np.zeros((V, dE_rows.shape[1]), dtype=np.float64)

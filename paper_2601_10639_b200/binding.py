@@ -28,7 +28,7 @@ FLAG_SINGLE_CTA = 2
 EXPORTS = (
     "stem_version", "stem_status_string", "stem_workspace_bytes", "stem_init_workspace",
     "stem_query_status", "stem_dedup_ids", "stem_ffn_forward", "stem_ffn_backward",
-    "stem_prefetch_rows", "stem_prefetch_rows_hot", "stem_lfu_workspace_bytes", "stem_lfu_touch", "stem_lfu_refresh", "stem_writeback_rows", "stem_writeback_rows_dma", "stem_gemm_bf16", "stem_step_arena_bytes",
+    "stem_dagger_forward", "stem_dagger_backward", "stem_prefetch_rows", "stem_prefetch_rows_hot", "stem_lfu_workspace_bytes", "stem_lfu_touch", "stem_lfu_refresh", "stem_writeback_rows", "stem_writeback_rows_dma", "stem_gemm_bf16", "stem_step_arena_bytes",
     "stem_ffn_step_host", "stem_ffn_step_host_flush", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
     "stem_dedup_ids_static", "stem_dedup_static_max_tokens",
 )
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
             "stem_dedup_ids": [shp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
             "stem_ffn_forward": [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
             "stem_ffn_backward": [shp] + [vp] * 17 + [sz, vp],
+            "stem_dagger_forward": [shp] + [vp] * 11 + [sz, vp],
+            "stem_dagger_backward": [shp] + [vp] * 17 + [sz, vp],
             "stem_prefetch_rows": [shp, vp, vp, vp, vp, vp, vp],
             "stem_prefetch_rows_hot": [shp, vp, vp, vp, vp, vp, vp, vp, vp, vp],
             "stem_lfu_workspace_bytes": [i32, i32, ctypes.POINTER(sz)],
@@ -163,6 +165,20 @@ def stem_ffn_backward(shape, dy, x, ids, W_gate, E, W_down, G_save, H_save, perm
                                    _p(dW_gate), _p(dW_down), _p(dE_rows), _p(unique_ids), _p(ws),
                                    ws.numel() * ws.element_size(), _stream(stream)),
            "stem_ffn_backward")
+
+
+def stem_dagger_forward(shape, x, ids, W_gate, W_up, E, W_down, y, G_save, H_save, U_save, ws, stream=None) -> None:
+    _check(lib().stem_dagger_forward(ctypes.byref(shape), _p(x), _p(ids), _p(W_gate), _p(W_up), _p(E), _p(W_down), _p(y),
+                                     _p(G_save), _p(H_save), _p(U_save), _p(ws), ws.numel() * ws.element_size(),
+                                     _stream(stream)), "stem_dagger_forward")
+
+
+def stem_dagger_backward(shape, dy, x, W_gate, W_up, W_down, G_save, H_save, U_save, perm, seg_offsets, n_unique,
+                         dx, dW_gate, dW_up, dW_down, dE_rows, ws, stream=None) -> None:
+    _check(lib().stem_dagger_backward(ctypes.byref(shape), _p(dy), _p(x), _p(W_gate), _p(W_up), _p(W_down), _p(G_save),
+                                      _p(H_save), _p(U_save), _p(perm), _p(seg_offsets), _p(n_unique), _p(dx),
+                                      _p(dW_gate), _p(dW_up), _p(dW_down), _p(dE_rows), _p(ws),
+                                      ws.numel() * ws.element_size(), _stream(stream)), "stem_dagger_backward")
 
 
 def stem_prefetch_rows(shape, ids, n_ids, table, dev_cache, ws, stream=None) -> None:

@@ -325,6 +325,110 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
   return STEM_OK;
 }
 
+// ---- STEM-dagger: the up-projection is kept and the table row is added to its output -------
+int stem_dagger_forward(const stem_shape_t* shape, const void* x, const int32_t* ids, const void* W_gate,
+                        const void* W_up, const void* E, const void* W_down, void* y, void* G_save, void* H_save,
+                        void* U_save, void* ws, size_t ws_bytes, void* stream) {
+  if (int rc = check_shape(shape)) return rc;
+  if (!ws || !aligned16(ws)) return STEM_ERR_INVALID_ARG;
+  if (shape->T == 0) return STEM_OK;
+  if (!x || !ids || !W_gate || !W_up || !E || !W_down || !y || !U_save) return STEM_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(W_gate) || !aligned16(W_up) || !aligned16(E) || !aligned16(W_down) || !aligned16(y) ||
+      !aligned16(G_save) || !aligned16(H_save) || !aligned16(U_save))
+    return STEM_ERR_INVALID_ARG;
+  const WsLayout w = ws_layout(shape);
+  if (ws_bytes < w.total) return STEM_ERR_WORKSPACE_TOO_SMALL;
+  if (use_tc(shape) && !is_sm100()) return STEM_ERR_UNSUPPORTED_ARCH;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int T = shape->T, d = shape->d_model, F = shape->d_ff;
+  void* H = H_save ? H_save : static_cast<char*>(ws) + w.h_off;
+  cudaError_t e;
+  {  // U = x W_up^T + E[ids]: the lookup is added in the up GEMM's epilogue
+    EpiParams up;
+    up.ids = ids; up.E = E; up.V = shape->V; up.H = U_save; up.status = status_of(ws);
+    ProfScope prof("up_gemm", st);
+    e = gemm(shape, T, F, d, x, false, W_up, false, kEpiAdd, up, st);
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+  {  // G = x W_gate^T, H = SiLU(G) (.) U: the gate epilogue with U as a [T, d_ff] "table" indexed by position
+    EpiParams gate;
+    gate.ids = nullptr; gate.E = U_save; gate.V = T; gate.H = H; gate.G = G_save; gate.status = status_of(ws);
+    ProfScope prof("gate_gemm", st);
+    e = gemm(shape, T, F, d, x, false, W_gate, false, kEpiGate, gate, st);
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+  EpiParams down;
+  down.out = y; down.out_fp32 = shape->dtype == STEM_DTYPE_FP32; down.status = status_of(ws);
+  down.sk_scratch = static_cast<char*>(ws) + w.sk_off; down.sk_bytes = w.sk_bytes;
+  {
+    ProfScope prof("down_gemm", st);
+    e = gemm(shape, T, d, F, H, false, W_down, false, kEpiStore, down, st);
+  }
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
+int stem_dagger_backward(const stem_shape_t* shape, const void* dy, const void* x, const void* W_gate,
+                         const void* W_up, const void* W_down, const void* G_save, const void* H_save,
+                         const void* U_save, const int32_t* perm, const int32_t* seg_offsets,
+                         const int32_t* n_unique, void* dx, void* dW_gate, void* dW_up, void* dW_down, void* dE_rows,
+                         void* ws, size_t ws_bytes, void* stream) {
+  if (int rc = check_shape(shape)) return rc;
+  if (!ws || !aligned16(ws)) return STEM_ERR_INVALID_ARG;
+  if (shape->T == 0) return STEM_OK;
+  if (!dy || !x || !W_gate || !W_up || !W_down || !G_save || !U_save) return STEM_ERR_INVALID_ARG;
+  if (dW_down && !H_save) return STEM_ERR_INVALID_ARG;
+  if (dE_rows && (!perm || !seg_offsets || !n_unique)) return STEM_ERR_INVALID_ARG;
+  if (!aligned16(dy) || !aligned16(x) || !aligned16(W_gate) || !aligned16(W_up) || !aligned16(W_down) ||
+      !aligned16(G_save) || !aligned16(H_save) || !aligned16(U_save) || !aligned16(dx) || !aligned16(dW_gate) ||
+      !aligned16(dW_up) || !aligned16(dW_down) || !aligned16(dE_rows))
+    return STEM_ERR_INVALID_ARG;
+  const WsLayout w = ws_layout(shape);
+  if (ws_bytes < w.total) return STEM_ERR_WORKSPACE_TOO_SMALL;
+  if (use_tc(shape) && !is_sm100()) return STEM_ERR_UNSUPPORTED_ARCH;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int T = shape->T, d = shape->d_model, F = shape->d_ff;
+  const int grad_fp32 = shape->grad_dtype == STEM_DTYPE_FP32;
+  char* base = static_cast<char*>(ws);
+  void* dU = base + w.du_off;
+  void* dG = base + w.dg_off;
+  cudaError_t e;
+  {  // dH = dy W_down; dU = dH SiLU(G) (gradient of U = W_up x + E[ids]); dG = dH U SiLU'(G)
+    EpiParams dh;
+    dh.ids = nullptr; dh.E = U_save; dh.V = T; dh.H = dU; dh.G = dG; dh.Gin = G_save; dh.status = status_of(ws);
+    ProfScope prof("dh_gemm", st);
+    e = gemm(shape, T, F, d, dy, false, W_down, true, kEpiDH, dh, st);
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+  auto grad = [&](const char* name, void* out, int M, int N, const void* A, const void* Bm) {
+    EpiParams p; p.out = out; p.out_fp32 = grad_fp32; p.status = status_of(ws);
+    p.sk_scratch = base + w.sk_off; p.sk_bytes = w.sk_bytes;
+    ProfScope prof(name, st);
+    return gemm(shape, M, N, T, A, true, Bm, true, kEpiStore, p, st);   // contraction over the tokens
+  };
+  if (dW_down && (e = grad("dw_down_gemm", dW_down, d, F, dy, H_save)) != cudaSuccess) return cuda_fail(e);
+  if (dE_rows) {
+    ProfScope prof("seg_reduce", st);
+    e = launch_segreduce(T, F, shape->dtype, shape->grad_dtype, dU, perm, seg_offsets, n_unique, dE_rows,
+                         base + w.part_off, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  if (dW_gate && (e = grad("dw_gate_gemm", dW_gate, F, d, dG, x)) != cudaSuccess) return cuda_fail(e);
+  if (dW_up && (e = grad("dw_up_gemm", dW_up, F, d, dU, x)) != cudaSuccess) return cuda_fail(e);
+  if (dx) {  // dx = dG W_gate + dU W_up: the second product is added onto the first in its epilogue
+    EpiParams p; p.out = dx; p.out_fp32 = shape->dtype == STEM_DTYPE_FP32; p.status = status_of(ws);
+    {
+      ProfScope prof("dx_gemm", st);
+      e = gemm(shape, T, d, F, dG, false, W_gate, true, kEpiStore, p, st);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    EpiParams a; a.ids = nullptr; a.E = dx; a.V = T; a.H = dx; a.status = status_of(ws);
+    ProfScope prof("dx_up_gemm", st);
+    e = gemm(shape, T, d, F, dU, false, W_up, true, kEpiAdd, a, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  return STEM_OK;
+}
+
 int stem_prefetch_rows(const stem_shape_t* shape, const int32_t* ids, const int32_t* n_ids, const void* table,
                        void* dev_cache, void* ws, void* stream) {
   if (int rc = check_shape(shape)) return rc;

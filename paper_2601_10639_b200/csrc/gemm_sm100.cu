@@ -131,6 +131,12 @@ __device__ __forceinline__ void epilogue_row32(const EpiParams& ep, uint32_t buf
       for (int i = 0; i < 16; ++i) o[i] = pack_bf16(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
       stage_row_bf16(buf, lane, o);
     }
+  } else if (KIND == kEpiAdd) {
+    uint32_t o[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+      o[i] = pack_bf16(__uint_as_float(acc[2 * i]) + bf16_lo(e[i]), __uint_as_float(acc[2 * i + 1]) + bf16_hi(e[i]));
+    stage_row_bf16(buf, lane, o);
   } else if (KIND == kEpiGate) {
     uint32_t h[16], go[16];
 #pragma unroll
@@ -231,7 +237,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
     ptx::prefetch_tensormap(&tmC0);
-    if (KIND != kEpiStore) ptx::prefetch_tensormap(&tmC1);
+    if (KIND == kEpiGate || KIND == kEpiDH) ptx::prefetch_tensormap(&tmC1);
   }
   if (warp == 1) {
     if (CTAS == 2) {
@@ -364,7 +370,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const __nv_bfloat16* e_row = nullptr;
       const __nv_bfloat16* g_row = nullptr;
       if (KIND != kEpiStore && row_ok) {
-        int id = ep.ids[m];
+        int id = ep.ids != nullptr ? ep.ids[m] : m;
         if (id < 0 || id >= ep.V) {
           report_error(ep.status, STEM_ERR_ID_RANGE, m);
           id = id < 0 ? 0 : ep.V - 1;
@@ -670,9 +676,11 @@ cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const 
   //                   dW_down / dW_gate (MN,MN,store); the plain-GEMM entry adds (MN,K,store)
   if (!a_mn && !b_mn) {
     if (kind == kEpiGate) return launch_ctas<false, false, kEpiGate>(A, B, M, N, K, ep, pair, stream);
+    if (kind == kEpiAdd) return launch_ctas<false, false, kEpiAdd>(A, B, M, N, K, ep, pair, stream);
     if (kind == kEpiStore) return launch_ctas<false, false, kEpiStore>(A, B, M, N, K, ep, pair, stream);
   } else if (!a_mn && b_mn) {
     if (kind == kEpiDH) return launch_ctas<false, true, kEpiDH>(A, B, M, N, K, ep, pair, stream);
+    if (kind == kEpiAdd) return launch_ctas<false, true, kEpiAdd>(A, B, M, N, K, ep, pair, stream);
     if (kind == kEpiStore) return launch_ctas<false, true, kEpiStore>(A, B, M, N, K, ep, pair, stream);
   } else if (a_mn && b_mn) {
     if (kind == kEpiStore) return launch_ctas<true, true, kEpiStore>(A, B, M, N, K, ep, pair, stream);

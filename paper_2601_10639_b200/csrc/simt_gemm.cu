@@ -17,6 +17,9 @@ __device__ __forceinline__ void epilogue_elem(const EpiParams& ep, int m, int n,
   if (KIND == kEpiStore) {
     if (ep.out_fp32) static_cast<float*>(ep.out)[o] = acc;
     else static_cast<T*>(ep.out)[o] = from_f32<T>(acc);
+  } else if (KIND == kEpiAdd) {
+    const float u = to_f32(static_cast<const T*>(ep.E)[static_cast<size_t>(row_id) * N + n]);
+    static_cast<T*>(ep.H)[o] = from_f32<T>(acc + u);
   } else if (KIND == kEpiGate) {
     const float u = to_f32(static_cast<const T*>(ep.E)[static_cast<size_t>(row_id) * N + n]);
     const float s = sigmoid_f32(acc);
@@ -90,7 +93,7 @@ simt_gemm_kernel(int M, int N, int K, const T* __restrict__ A, const T* __restri
     if (m >= M) continue;
     int row_id = 0;
     if (KIND != kEpiStore) {
-      row_id = ep.ids[m];
+      row_id = ep.ids != nullptr ? ep.ids[m] : m;
       if (row_id < 0 || row_id >= ep.V) {
         report_error(ep.status, STEM_ERR_ID_RANGE, m);
         row_id = row_id < 0 ? 0 : ep.V - 1;
@@ -114,6 +117,7 @@ cudaError_t launch_kind(int M, int N, int K, const void* A, const void* B, EpiKi
     case kEpiStore: simt_gemm_kernel<T, A_MN, B_MN, kEpiStore><<<grid, 256, 0, stream>>>(M, N, K, a, b, ep); break;
     case kEpiGate: simt_gemm_kernel<T, A_MN, B_MN, kEpiGate><<<grid, 256, 0, stream>>>(M, N, K, a, b, ep); break;
     case kEpiDH: simt_gemm_kernel<T, A_MN, B_MN, kEpiDH><<<grid, 256, 0, stream>>>(M, N, K, a, b, ep); break;
+    case kEpiAdd: simt_gemm_kernel<T, A_MN, B_MN, kEpiAdd><<<grid, 256, 0, stream>>>(M, N, K, a, b, ep); break;
   }
   count_launches(1);
   return cudaGetLastError();

@@ -36,7 +36,7 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
 __device__ __forceinline__ float sigmoid_f32(float g) { return 1.0f / (1.0f + expf(-g)); }
 
 // ---- epilogue descriptions (shared by the FMA and the tensor-core GEMM front ends) ---
-enum EpiKind : int { kEpiStore = 0, kEpiGate = 1, kEpiDH = 2 };
+enum EpiKind : int { kEpiStore = 0, kEpiGate = 1, kEpiDH = 2, kEpiAdd = 3 };
 
 struct EpiParams {
   // kEpiStore: out[m*ld + n] = acc              (out_fp32 selects fp32 or bf16/T storage)
@@ -45,6 +45,8 @@ struct EpiParams {
   // kEpiGate:  g = acc; H = SiLU(g) * E[ids[m], n]; optional G = g
   // kEpiDH:    dh = acc; g = G[m,n]; u = E[ids[m], n];
   //            dU = dh * SiLU(g); dG = dh * u * SiLU'(g)
+  // kEpiAdd:   H[m,n] = acc + E[ids[m], n]      (bf16/T storage; in place when E == H)
+  // ids == nullptr in kEpiGate / kEpiDH / kEpiAdd means ids[m] = m: E is then a [M,N] matrix
   const int32_t* ids = nullptr;
   const void* E = nullptr;
   int V = 0;

@@ -428,6 +428,41 @@ def test_prefetch_with_hot_set_and_prefill_stack():
             assert stack.stats.tolist() == [2 * L * n_hot, 2 * L * (n_u - n_hot)]
 
 
+@pytest.mark.parametrize("dtype_code,flags,tol", [(B.DTYPE_BF16, 0, TOL_BF16), (B.DTYPE_BF16, B.FLAG_SIMT, TOL_BF16),
+                                                   (B.DTYPE_FP32, 0, TOL_FP32)], ids=["tcgen05", "fma_bf16", "fp32"])
+def test_dagger_variant(dtype_code, flags, tol):
+    """STEM-dagger, forward and backward, against the checker (ragged sizes, repeated ids)."""
+    w = synth.Workload("t", 700, 264, 520, 900, "bf16" if dtype_code == B.DTYPE_BF16 else "fp32", "zipf")
+    inp = synth.make_inputs(w, seed=120)
+    W_up_np = synth.normal(120, 9, (w.d_ff, w.d_model), w.d_model ** -0.5)
+    if dtype_code == B.DTYPE_BF16:
+        W_up_np = synth.round_bf16(W_up_np)
+    st = runner.state_from_numpy(inp, dtype_code, w.V, flags=flags)
+    W_up = runner.to_device(W_up_np, dtype_code)
+    b = st.bufs
+    dt = runner.torch_dtype(dtype_code)
+    U = torch.empty(w.T, w.d_ff, dtype=dt, device="cuda")
+    dW_up = torch.empty(w.d_ff, w.d_model, dtype=torch.float32, device="cuda")
+    st.dedup()
+    B.stem_dagger_forward(st.shape, st.x, st.ids, st.W_gate, W_up, st.E, st.W_down, b["y"], b["G"], b["H"], U, b["ws"])
+    B.stem_dagger_backward(st.shape, st.dy, st.x, st.W_gate, W_up, st.W_down, b["G"], b["H"], U, b["perm"],
+                           b["seg_offsets"], b["n_unique"], b["dx"], b["dW_gate"], dW_up, b["dW_down"], b["dE_rows"],
+                           b["ws"])
+    torch.cuda.synchronize()
+    assert st.status() == B.OK
+    y_ref, im = O.dagger_forward(inp["x"], inp["ids"], inp["W_gate"], W_up_np, inp["E"], inp["W_down"], True)
+    bw = O.dagger_backward(inp["dy"], inp["x"], inp["ids"], inp["W_gate"], W_up_np, inp["E"], inp["W_down"])
+    n_u = int(b["n_unique"].item())
+    errs = {"U": O.scaled_max_err(_np(U), im["U"]), "H": O.scaled_max_err(_np(b["H"]), im["H"]),
+            "y": O.scaled_max_err(_np(b["y"]), y_ref), "dx": O.scaled_max_err(_np(b["dx"]), bw["dx"]),
+            "dW_gate": O.scaled_max_err(_np(b["dW_gate"]), bw["dW_gate"]),
+            "dW_up": O.scaled_max_err(_np(dW_up), bw["dW_up"]),
+            "dW_down": O.scaled_max_err(_np(b["dW_down"]), bw["dW_down"]),
+            "dE_rows": O.scaled_max_err(_np(b["dE_rows"][:n_u]), bw["dE_rows"])}
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, (bad, errs)
+
+
 def test_lfu_cache_tracks_the_most_frequent_ids():
     """Decode steps of Zipfian ids: after every refresh the cache holds exactly the checker's top-K
     set, every cached row equals its table row, slots are consistent, and the hit counters equal

@@ -334,3 +334,49 @@ def test_lfu_hot_set_against_brute_force():
             assert all(freq[i] <= inside_min for i in range(V) if i not in picked)
     ids = np.array([1, 1, 5, 7, 7, 7, 2])
     assert O.lfu_hits(ids, [7, 1]) == 5 and O.lfu_hits(ids, []) == 0
+
+
+# ---------------------------------------------------------------------------------------
+# STEM-dagger (Appendix): W_up x + U[t] in place of U[t]
+# ---------------------------------------------------------------------------------------
+def test_dagger_reduces_to_dense_swiglu_autograd_and_to_the_layer():
+    """Dense SwiGLU on [x ; onehot(id)] with W_u' = [W_up  E^T] is STEM-dagger (torch autograd gives
+    every gradient); W_up = 0 gives the layer itself; E = 0 gives the plain dense block."""
+    c = _rand_case(19, 6, 10, 5, seed=11)
+    rng = np.random.default_rng(12)
+    W_up = rng.normal(size=(10, 6)) / np.sqrt(6)
+    T, d = c["x"].shape
+    V, F = c["E"].shape
+    x = torch.tensor(c["x"], requires_grad=True)
+    Wg = torch.tensor(c["W_gate"], requires_grad=True)
+    Wu = torch.tensor(W_up, requires_grad=True)
+    Wd = torch.tensor(c["W_down"], requires_grad=True)
+    Et = torch.tensor(c["E"].T.copy(), requires_grad=True)
+    onehot = torch.nn.functional.one_hot(torch.tensor(c["ids"], dtype=torch.int64), V).to(torch.float64)
+    xa = torch.cat([x, onehot], dim=1)
+    Wg_aug = torch.cat([Wg, torch.zeros(F, V, dtype=torch.float64)], dim=1)
+    Wu_aug = torch.cat([Wu, Et], dim=1)
+    lin = torch.nn.functional.linear
+    y = lin(torch.nn.functional.silu(lin(xa, Wg_aug)) * lin(xa, Wu_aug), Wd)
+    (y * torch.tensor(c["dy"])).sum().backward()
+    got_y = O.dagger_forward(c["x"], c["ids"], c["W_gate"], W_up, c["E"], c["W_down"])
+    b = O.dagger_backward(c["dy"], c["x"], c["ids"], c["W_gate"], W_up, c["E"], c["W_down"])
+    kw = dict(rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(got_y, y.detach().numpy(), **kw)
+    np.testing.assert_allclose(b["dx"], x.grad.numpy(), **kw)
+    np.testing.assert_allclose(b["dW_gate"], Wg.grad.numpy(), **kw)
+    np.testing.assert_allclose(b["dW_up"], Wu.grad.numpy(), **kw)
+    np.testing.assert_allclose(b["dW_down"], Wd.grad.numpy(), **kw)
+    np.testing.assert_allclose(O.dE_dense(b["unique_ids"], b["dE_rows"], V), Et.grad.numpy().T, **kw)
+    # W_up = 0: the layer itself, forward and every shared gradient
+    z = np.zeros_like(W_up)
+    np.testing.assert_allclose(O.dagger_forward(c["x"], c["ids"], c["W_gate"], z, c["E"], c["W_down"]),
+                               O.forward(c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"]), **kw)
+    b0 = O.dagger_backward(c["dy"], c["x"], c["ids"], c["W_gate"], z, c["E"], c["W_down"])
+    b1 = O.backward(c["dy"], c["x"], c["ids"], c["W_gate"], c["E"], c["W_down"])
+    for k in ("dx", "dW_gate", "dW_down", "dE_rows"):
+        np.testing.assert_allclose(b0[k], b1[k], **kw)
+    # E = 0: a plain SwiGLU block (Background, Eq. 1), written out directly
+    y_dense = (O.silu(c["x"] @ c["W_gate"].T) * (c["x"] @ W_up.T)) @ c["W_down"].T
+    np.testing.assert_allclose(O.dagger_forward(c["x"], c["ids"], c["W_gate"], W_up, np.zeros_like(c["E"]), c["W_down"]),
+                               y_dense, **kw)
