@@ -541,6 +541,8 @@ def main():
                     help="prefill workload: sizes of the on-device hot set to try")
     ap.add_argument("--unique-growth", action="store_true", help="print distinct rows vs context length and exit")
     ap.add_argument("--grad-bf16", action="store_true", help="host-table workload: bf16 weight and table gradients")
+    ap.add_argument("--variant", default="stem", choices=["stem", "dagger"],
+                    help="dagger: the paper's STEM-dagger ablation (up-projection kept, table row added)")
     ap.add_argument("--no-profile", action="store_true",
                     help="do not record per-step events inside the timed region (checks what they cost)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
@@ -602,6 +604,24 @@ def main():
     st.ids = torch.from_numpy(ids_np).to(dev)
     st.allocate(backward)
     stream = torch.cuda.current_stream()
+    flops_step = layer_flops(T, d, F, backward)
+    run_step = lambda: st.step(backward=backward)
+    if args.variant == "dagger":
+        # STEM-dagger (Appendix): the up-projection is kept; 3 contractions forward, 6 backward
+        W_up = (torch.randn(F, d, generator=gen, device=dev, dtype=torch.float32) * d ** -0.5).to(dt)
+        U = torch.empty(T, F, dtype=dt, device=dev)
+        dW_up = torch.empty(F, d, dtype=torch.float32, device=dev)
+        flops_step = (18.0 if backward else 6.0) * T * d * F
+        b_ = st.bufs
+
+        def run_step():
+            st.dedup()
+            B.stem_dagger_forward(st.shape, st.x, st.ids, st.W_gate, W_up, st.E, st.W_down, b_["y"], b_["G"], b_["H"], U,
+                                  b_["ws"])
+            if backward:
+                B.stem_dagger_backward(st.shape, st.dy, st.x, st.W_gate, W_up, st.W_down, b_["G"], b_["H"], U, b_["perm"],
+                                       b_["seg_offsets"], b_["n_unique"], b_["dx"], b_["dW_gate"], dW_up, b_["dW_down"],
+                                       b_["dE_rows"], b_["ws"])
 
     def barrier():
         if world > 1:
@@ -610,7 +630,7 @@ def main():
 
     # ---- device-resident timing ------------------------------------------------------------
     for _ in range(args.warmup):
-        st.step(backward=backward)
+        run_step()
     barrier()
     assert st.status() == B.OK, B.status_string(st.status())
     n_u = int(st.bufs["n_unique"].item())
@@ -622,7 +642,7 @@ def main():
         t0 = time.time()
         ev0.record(stream)
         for _ in range(args.steps):
-            st.step(backward=backward)
+            run_step()
         ev1.record(stream)
         barrier()
         t1 = time.time()
@@ -636,7 +656,7 @@ def main():
     # ---- end to end through the host-buffer entry point -------------------------------------
     esz = 2 if dcode == B.DTYPE_BF16 else 4
     e2e = None
-    if backward and not args.no_e2e:
+    if backward and not args.no_e2e and args.variant == "stem":
         hx, hdy = st.x.cpu().pin_memory(), st.dy.cpu().pin_memory()
         hids = st.ids.cpu().pin_memory()
         hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
@@ -757,10 +777,10 @@ def main():
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if dcode == B.DTYPE_BF16 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "T": T, "d_model": d, "d_ff": F, "V": V, "ids": w.id_dist,
-                   "n_unique": n_u, "backward": backward, "parallelism": f"replicas x{world}",
+                   "n_unique": n_u, "backward": backward, "variant": args.variant, "parallelism": f"replicas x{world}",
                    "l2": "per-step working set (~2.5 GB at 1b shapes) exceeds the 126 MB L2; no flush"},
         "gpu_launches": int(launches),
-        "tflops_step": layer_flops(T, d, F, backward) / (ms_per_step * 1e-3) / 1e12,
+        "tflops_step": flops_step / (ms_per_step * 1e-3) / 1e12,
         "clocks": clock_summary,
         "roofline": roofline,
         "kernels": kernels,
