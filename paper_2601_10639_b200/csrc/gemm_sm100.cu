@@ -559,12 +559,11 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
   using L = Smem<BN, STAGES, CTAS>;
   static_assert(L::kTotal <= 232448, "exceeds the shared memory a CTA can have");
   auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES, WIDE, CTAS>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static PerDeviceOnce configured;
+  if (cudaError_t ce = configured.run([&] {
+        return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+      }))
+    return ce;
   // persistent: one CTA (or one pair) per SM (pair of SMs), each walking its work list
   const int tiles_m = (M + BM * CTAS - 1) / (BM * CTAS), tiles_n = (N + BN - 1) / BN;
   const int units = tiles_m * tiles_n;

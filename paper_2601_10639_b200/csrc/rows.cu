@@ -101,8 +101,8 @@ cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int3
   int blocks = (max_rows + rows_per_cta - 1) / rows_per_cta;
   const int cap = table_on_host ? kHostLinkCtas : device_sm_count() * 8;
   if (blocks > cap) blocks = cap;
-  static const cudaError_t configured = prefer_max_shared(gather_rows_kernel);
-  if (configured != cudaSuccess) return configured;
+  static PerDeviceOnce configured;
+  if (cudaError_t ce = configured.run([] { return prefer_max_shared(gather_rows_kernel); })) return ce;
   gather_rows_kernel<<<blocks, threads, 0, stream>>>(V, vec, ids, n_ids, static_cast<const uint4*>(table),
                                                     static_cast<const uint4*>(hot_rows), hot_slot,
                                                     static_cast<uint4*>(dst), status, stats);
@@ -116,8 +116,8 @@ cudaError_t launch_writeback_rows(int max_rows, size_t row_bytes, const void* ro
   if (max_rows <= 0) return cudaSuccess;
   const int vec = static_cast<int>(row_bytes / 16);
   const int blocks = kHostLinkCtas;
-  static const cudaError_t configured = prefer_max_shared(writeback_rows_kernel);
-  if (configured != cudaSuccess) return configured;
+  static PerDeviceOnce configured;
+  if (cudaError_t ce = configured.run([] { return prefer_max_shared(writeback_rows_kernel); })) return ce;
   writeback_rows_kernel<<<blocks, kHostLinkThreads, 0, stream>>>(vec, static_cast<const uint4*>(rows), unique_ids,
                                                         n_rows, static_cast<uint4*>(host_rows), host_ids, host_n);
   count_launches(1);

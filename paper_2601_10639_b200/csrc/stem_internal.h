@@ -112,6 +112,22 @@ cudaError_t launch_lfu_refresh(int V, int K, size_t row_bytes, const int32_t* fr
                                void* scratch, cudaStream_t stream);
 
 int device_sm_count();
+
+// Function attributes (shared-memory size, preferred split) are per device: `done` is a
+// per-call-site table that remembers on which devices `set()` has already succeeded.
+struct PerDeviceOnce {
+  bool done[64] = {};
+  template <typename F> cudaError_t run(F set) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (done[dev]) return cudaSuccess;
+    e = set();
+    if (e == cudaSuccess) done[dev] = true;
+    return e;
+  }
+};
 void count_launches(int n);  // bookkeeping for stem_launch_count()
 
 }  // namespace stem
