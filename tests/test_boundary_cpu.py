@@ -78,6 +78,41 @@ def test_null_and_misaligned_arguments_are_rejected_on_the_host():
     assert L.stem_gemm_bf16(8, 8, 8, None, 0, None, 0, None, 0, 0, None, None) == B.ERR_INVALID_ARG
 
 
+def test_later_entry_points_reject_bad_arguments_on_the_host():
+    """Row cache, hot-set prefetch, copy-engine write-back, STEM-dagger, host-buffer step: the checks
+    that need no device run before any CUDA call."""
+    L = B.lib()
+    s = B.make_shape(16, 8, 8, 8)
+    sz = ctypes.c_size_t(0)
+    assert L.stem_lfu_workspace_bytes(100, 0, ctypes.byref(sz)) == B.ERR_INVALID_ARG          # K < 1
+    assert L.stem_lfu_workspace_bytes(100, 101, ctypes.byref(sz)) == B.ERR_INVALID_ARG        # K > V
+    assert L.stem_lfu_workspace_bytes(100, 10, None) == B.ERR_INVALID_ARG
+    assert L.stem_lfu_workspace_bytes(32000, 2048, ctypes.byref(sz)) == B.OK and sz.value > 32000 * 4 * 5
+    assert L.stem_lfu_touch(-1, 10, None, None, None, None, None) == B.ERR_INVALID_ARG
+    assert L.stem_lfu_touch(0, 10, None, None, None, None, None) == B.OK                       # nothing to count
+    assert L.stem_lfu_touch(4, 10, None, 0x1000, 0x1000, None, None) == B.ERR_INVALID_ARG
+    assert L.stem_lfu_refresh(ctypes.byref(s), 9, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, None, 0x1000, 1 << 20,
+                              None) == B.ERR_INVALID_ARG                                       # K > V
+    assert L.stem_lfu_refresh(ctypes.byref(s), 4, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, None, 0x1000, 16,
+                              None) == B.ERR_WORKSPACE_TOO_SMALL
+    assert L.stem_prefetch_rows_hot(ctypes.byref(s), 0x1000, 0x1000, 0x1000, None, 0x1000, 0x1000, None, None,
+                                    None) == B.ERR_INVALID_ARG                                 # no hot rows
+    assert L.stem_writeback_rows_dma(ctypes.byref(s), 0x1000, 0x1000, 9, 0x1000, 0x1000, None) == B.ERR_INVALID_ARG
+    assert L.stem_writeback_rows_dma(ctypes.byref(s), 0x1000, 0x1000, 0, 0x1000, 0x1000, None) == B.OK   # no rows
+    args = [ctypes.byref(s)] + [None] * 11 + [0, None]
+    assert L.stem_dagger_forward(*args) == B.ERR_INVALID_ARG
+    args = [ctypes.byref(s)] + [None] * 17 + [0, None]
+    assert L.stem_dagger_backward(*args) == B.ERR_INVALID_ARG
+    bad = B.make_shape(16, 8, 12, 8)
+    args = [ctypes.byref(bad)] + [0x1000] * 11 + [1 << 30, None]
+    assert L.stem_dagger_forward(*args) == B.ERR_UNSUPPORTED_SHAPE
+    args = [ctypes.byref(s)] + [None] * 15 + [0, None]
+    assert L.stem_ffn_step_host(*args) == B.ERR_INVALID_ARG
+    assert L.stem_step_arena_bytes(ctypes.byref(s), ctypes.byref(sz)) == B.OK and sz.value > 0
+    for code in (B.OK, B.ERR_STATIC_LIMIT):
+        assert B.status_string(code)
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "libstem.so"))
