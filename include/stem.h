@@ -18,7 +18,7 @@
  *     device memory.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
  *     only enqueue work; they do not synchronise unless stated.
- *   - Outputs are overwritten, never accumulated into.
+ *   - Outputs are overwritten, except the weight gradients under STEM_FLAG_ACCUM_GRADS.
  *   - Return value: STEM_OK or a negative STEM_ERR_* code.  Conditions only the device
  *     can see (an id outside [0,V), a pipeline wait that ran out) are recorded in the
  *     workspace's status word and read back with stem_query_status().  A bad id is
@@ -56,6 +56,12 @@ extern "C" {
 
 #define STEM_FLAG_SIMT 1 /* run the bf16 contractions on the plain-FMA kernels (debug aid) */
 #define STEM_FLAG_SINGLE_CTA 2 /* tensor-core contractions on single CTAs instead of CTA pairs (debug aid) */
+/* Backward adds the weight gradients (dW_gate, dW_down, and dW_up of the dagger variant) to what
+ * the caller's buffers hold instead of overwriting them: gradient accumulation over
+ * micro-batches.  Not a step of the paper's method; dx and dE_rows are still overwritten (the
+ * rows of dE_rows belong to this call's unique ids).  With bf16 gradients the product is rounded
+ * to bf16 before the bf16 add. */
+#define STEM_FLAG_ACCUM_GRADS 4
 
 typedef struct {
   int32_t T;          /* positions in this call (batch x sequence)                 */

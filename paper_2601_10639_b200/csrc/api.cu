@@ -297,6 +297,7 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
   if (e != cudaSuccess) return cuda_fail(e);
   if (dW_down) {  // dW_down[i,j] = sum_t dy[t,i] H[t,j]
     EpiParams p; p.out = dW_down; p.out_fp32 = grad_fp32; p.status = status_of(ws);
+    p.accumulate = (shape->flags & STEM_FLAG_ACCUM_GRADS) != 0;
     p.sk_scratch = base + w.sk_off; p.sk_bytes = w.sk_bytes;
     ProfScope prof("dw_down_gemm", st);
     e = gemm(shape, d, F, T, dy, true, H_save, true, kEpiStore, p, st);
@@ -310,6 +311,7 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
   }
   if (dW_gate) {  // dW_gate[j,k] = sum_t dG[t,j] x[t,k]
     EpiParams p; p.out = dW_gate; p.out_fp32 = grad_fp32; p.status = status_of(ws);
+    p.accumulate = (shape->flags & STEM_FLAG_ACCUM_GRADS) != 0;
     p.sk_scratch = base + w.sk_off; p.sk_bytes = w.sk_bytes;
     ProfScope prof("dw_gate_gemm", st);
     e = gemm(shape, F, d, T, dG, true, x, true, kEpiStore, p, st);
@@ -401,6 +403,7 @@ int stem_dagger_backward(const stem_shape_t* shape, const void* dy, const void* 
   if (e != cudaSuccess) return cuda_fail(e);
   auto grad = [&](const char* name, void* out, int M, int N, const void* A, const void* Bm) {
     EpiParams p; p.out = out; p.out_fp32 = grad_fp32; p.status = status_of(ws);
+    p.accumulate = (shape->flags & STEM_FLAG_ACCUM_GRADS) != 0;
     p.sk_scratch = base + w.sk_off; p.sk_bytes = w.sk_bytes;
     ProfScope prof(name, st);
     return gemm(shape, M, N, T, A, true, Bm, true, kEpiStore, p, st);   // contraction over the tokens

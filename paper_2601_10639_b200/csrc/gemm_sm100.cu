@@ -431,7 +431,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           ptx::fence_proxy_async();
           __syncwarp();
           if (lane == 0 && m_warp < M && n < N) {
-            ptx::tma_store_2d(&tmC0, out_buf, n, m_warp);
+            if (KIND == kEpiStore && ep.accumulate) ptx::tma_reduce_add_2d(&tmC0, out_buf, n, m_warp);
+            else ptx::tma_store_2d(&tmC0, out_buf, n, m_warp);
             if (second_out) ptx::tma_store_2d(&tmC1, out_buf + 2048, n, m_warp);
             ptx::bulk_commit_group();
           }
@@ -476,7 +477,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 template <int BN, int CTAS>
 __global__ void __launch_bounds__(256)
 tail_fixup_kernel(int M, int N, int dp_tiles, int tail, int split, int tiles_m, int tiles_n, int group_m,
-                  const float* __restrict__ partial, void* __restrict__ out, int out_fp32) {
+                  const float* __restrict__ partial, void* __restrict__ out, int out_fp32, int accumulate) {
   constexpr int TM = BM * CTAS;
   ptx::grid_dependency_wait();
   ptx::grid_launch_dependents();
@@ -495,12 +496,19 @@ tail_fixup_kernel(int M, int N, int dp_tiles, int tail, int split, int tiles_m, 
     }
     const size_t o = static_cast<size_t>(m) * N + nn;   // N is a multiple of 8: 4 columns never straddle the edge
     if (out_fp32) {
-      *reinterpret_cast<float4*>(static_cast<float*>(out) + o) = acc;
+      float4* p = reinterpret_cast<float4*>(static_cast<float*>(out) + o);
+      if (accumulate) { const float4 v = *p; acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w; }
+      *p = acc;
     } else {
+      uint2* p = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + o);
+      if (accumulate) {
+        const uint2 v = *p;
+        acc.x += bf16_lo(v.x); acc.y += bf16_hi(v.x); acc.z += bf16_lo(v.y); acc.w += bf16_hi(v.y);
+      }
       uint2 pk;
       pk.x = pack_bf16(acc.x, acc.y);
       pk.y = pack_bf16(acc.z, acc.w);
-      *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + o) = pk;
+      *p = pk;
     }
   }
 }
@@ -594,7 +602,8 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     fcfg.attrs = attr + 1;
     fcfg.numAttrs = 1;
     e = cudaLaunchKernelEx(&fcfg, tail_fixup_kernel<BN, CTAS>, M, N, dp_tiles, sk_tail, sk_split, tiles_m, tiles_n, 8,
-                           static_cast<const float*>(ep.sk_scratch), ep.out, static_cast<int>(ep.out_fp32));
+                           static_cast<const float*>(ep.sk_scratch), ep.out, static_cast<int>(ep.out_fp32),
+                           static_cast<int>(ep.accumulate));
     count_launches(1);
   }
   return e != cudaSuccess ? e : cudaGetLastError();

@@ -15,8 +15,13 @@ __device__ __forceinline__ void epilogue_elem(const EpiParams& ep, int m, int n,
                                               float acc) {
   const size_t o = static_cast<size_t>(m) * N + n;
   if (KIND == kEpiStore) {
-    if (ep.out_fp32) static_cast<float*>(ep.out)[o] = acc;
-    else static_cast<T*>(ep.out)[o] = from_f32<T>(acc);
+    if (ep.out_fp32) {
+      float* p = static_cast<float*>(ep.out) + o;
+      *p = ep.accumulate ? *p + acc : acc;
+    } else {
+      T* p = static_cast<T*>(ep.out) + o;
+      *p = from_f32<T>(ep.accumulate ? to_f32(*p) + acc : acc);
+    }
   } else if (KIND == kEpiAdd) {
     const float u = to_f32(static_cast<const T*>(ep.E)[static_cast<size_t>(row_id) * N + n]);
     static_cast<T*>(ep.H)[o] = from_f32<T>(acc + u);

@@ -40,8 +40,10 @@ enum EpiKind : int { kEpiStore = 0, kEpiGate = 1, kEpiDH = 2, kEpiAdd = 3 };
 
 struct EpiParams {
   // kEpiStore: out[m*ld + n] = acc              (out_fp32 selects fp32 or bf16/T storage)
+  //            accumulate: out[m*ld + n] += acc   (gradient accumulation over micro-batches)
   void* out = nullptr;
   int out_fp32 = 0;
+  int accumulate = 0;
   // kEpiGate:  g = acc; H = SiLU(g) * E[ids[m], n]; optional G = g
   // kEpiDH:    dh = acc; g = G[m,n]; u = E[ids[m], n];
   //            dU = dh * SiLU(g); dG = dh * u * SiLU'(g)

@@ -180,6 +180,33 @@ def test_layer_bf16_grad_bf16():
     _full_parity(w, synth.make_inputs(w, seed=78), B.DTYPE_BF16, TOL_BF16, 0, grad_dtype=B.DTYPE_BF16)
 
 
+@pytest.mark.parametrize("flags", [0, B.FLAG_SINGLE_CTA, B.FLAG_SIMT], ids=["tcgen05_pair", "tcgen05_single", "fma"])
+@pytest.mark.parametrize("T,d,F,grad", [(600, 264, 520, B.DTYPE_FP32), (8192, 256, 512, B.DTYPE_FP32),
+                                        (8200, 264, 520, B.DTYPE_BF16)])
+def test_weight_gradients_accumulate_over_micro_batches(flags, T, d, F, grad):
+    """Two micro-batches, the second with the accumulate flag, against the checker's gradients of
+    the concatenated batch (the loss is a sum over positions, so its weight gradients add)."""
+    w = synth.Workload("t", T, d, F, 2000, "bf16", "zipf")
+    inputs = synth.make_inputs(w, seed=91)
+    bw = O.backward(inputs["dy"], inputs["x"], inputs["ids"], inputs["W_gate"], inputs["E"], inputs["W_down"])
+    cut = (T // 3) | 1          # uneven, odd split
+    acc = None
+    for lo, hi, fl in ((0, cut, flags), (cut, T, flags | B.FLAG_ACCUM_GRADS)):
+        part = {k: (v[lo:hi] if k in ("x", "dy", "ids") else v) for k, v in inputs.items()}
+        st = runner.state_from_numpy(part, B.DTYPE_BF16, w.V, grad_dtype=grad, flags=fl)
+        if acc is not None:
+            st.bufs["dW_gate"].copy_(acc[0]); st.bufs["dW_down"].copy_(acc[1])
+        else:
+            st.bufs["dW_gate"].fill_(7.0); st.bufs["dW_down"].fill_(-7.0)   # must be overwritten
+        st.step()
+        torch.cuda.synchronize()
+        assert st.status() == B.OK
+        acc = (st.bufs["dW_gate"].clone(), st.bufs["dW_down"].clone())
+    errs = {"dW_gate": O.scaled_max_err(_np(acc[0]), bw["dW_gate"]),
+            "dW_down": O.scaled_max_err(_np(acc[1]), bw["dW_down"])}
+    assert all(v <= TOL_BF16 for v in errs.values()), errs
+
+
 def test_backward_is_bitwise_reproducible():
     w = synth.Workload("t", 2048, 256, 1024, 500, "bf16", "zipf")
     st = runner.state_from_numpy(synth.make_inputs(w, seed=79), B.DTYPE_BF16, w.V)
