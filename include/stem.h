@@ -280,6 +280,48 @@ int stem_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t a_mn,
                    int32_t b_mn, void* C, int32_t c_fp32, int32_t flags, void* ws, void* stream);
 
 /*
+ * Table sharded over G GPUs (Section 3.4, "parallel embeddings": the table is always sharded
+ * across the available GPUs, whatever the backbone's parallelism; the cost is one exchange of
+ * the deduplicated rows, uniq(BL) x d_ff, Table 1).  The paper does not fix the row assignment;
+ * here GPU g owns the rows with id mod G == g and keeps row id at local index id / G.
+ *
+ * stem_shard_route turns a batch's distinct ids into the requests of that exchange:
+ *   send_local [n_max]  local row index asked of its owner, grouped by owner (owner 0 first),
+ *                       ascending id inside a group; entries [0, *n_unique) are written
+ *   send_slot  [n_max]  index into unique_ids of request j (where the answer's row, and later
+ *                       its gradient row, belongs)
+ *   send_counts [G]     requests per owner (device; the caller copies them to the host to size
+ *                       the exchange)
+ *   token_slot [T]      request whose answer is position t's row, or NULL: the layer is then
+ *                       run with ids = token_slot and E = the [n_unique, d_ff] rows as they
+ *                       came back, V = n_unique
+ * unique_ids [n_max], n_unique [1], inverse [T]: outputs of stem_dedup_ids (device).
+ * n_max >= *n_unique (normally min(T, V)); 1 <= G <= 1024.  route_ws: device scratch of
+ * stem_shard_route_workspace_bytes(n_max, G) bytes, 16-byte aligned.  Integer work only.
+ *
+ * stem_reduce_rows is the table-gradient reduce as a call of its own, for the owner's side of
+ * the return exchange: rows_out[r,:] = sum over the positions p of segment r of
+ * rows_in[perm[p],:], in a fixed order.  shape->T = rows received, shape->d_ff = row length,
+ * rows_in and rows_out in shape->grad_dtype; perm, seg_offsets, n_unique from stem_dedup_ids
+ * over the received local row indices; rows_out [min(T,V), d_ff]; ws as for
+ * stem_ffn_backward with this shape.
+ */
+/* The owner's side of the row exchange: out[r,:] = table[ids[r],:] for r < *n_ids, where ids
+ * may repeat (several GPUs may ask for the same row), so up to shape->T rows are written
+ * whatever shape->V is.  table [V,d_ff] and out [T,d_ff] in shape->dtype, device memory (or
+ * table in page-locked host memory); ids, n_ids: device; ws: any initialised workspace
+ * (status word only) or NULL. */
+int stem_gather_rows(const stem_shape_t* shape, const int32_t* ids, const int32_t* n_ids, const void* table,
+                     void* out, void* ws, void* stream);
+int stem_shard_route_workspace_bytes(int32_t n_max, int32_t G, size_t* bytes /*host, out*/);
+int stem_shard_route(int32_t n_max, int32_t T, int32_t G, const int32_t* unique_ids, const int32_t* n_unique,
+                     const int32_t* inverse, int32_t* send_local, int32_t* send_slot, int32_t* send_counts,
+                     int32_t* token_slot, void* route_ws, size_t route_ws_bytes, void* stream);
+int stem_reduce_rows(const stem_shape_t* shape, const void* rows_in, const int32_t* perm,
+                     const int32_t* seg_offsets, const int32_t* n_unique, void* rows_out, void* ws,
+                     size_t ws_bytes, void* stream);
+
+/*
  * One training step of the layer from host buffers (the composition of the calls above,
  * in the order Section 3.4 gives for training: ids deduplicated, forward, backward, table
  * gradients reduced per unique id):

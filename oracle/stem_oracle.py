@@ -16,6 +16,9 @@ It is deliberately unblocked and unfused so it can be read against the equations
               defined here: positions stably sorted by id, the distinct ids ascending,
               where each id's run starts, and each position's slot.
 
+* shard_route, shard_owner_gradient -- Section 3.4: the table sharded across GPUs; the row
+              assignment (id mod G) is this build's reading, the rest follows from it.
+
 SiLU is not defined in the paper; the standard SiLU(z) = z * sigmoid(z) is used.
 Token ids are 0-based.  There are no bias terms (Table 1 caption).
 
@@ -189,6 +192,36 @@ def lfu_hot_set(freq, K: int) -> np.ndarray:
 def lfu_hits(ids, hot_ids) -> int:
     """Lookups of one decode step that a cache holding `hot_ids` serves."""
     return int(np.isin(np.asarray(ids), np.asarray(hot_ids)).sum())
+
+
+def shard_route(unique_ids, G: int) -> dict:
+    """Requests of the row exchange for a table sharded over G GPUs (Section 3.4, "parallel
+    embeddings").  The paper does not say which GPU holds which row; the reading here is
+    owner = id mod G, local row index = id // G.  Requests are grouped by owner (owner 0
+    first) and keep ascending id inside a group."""
+    unique_ids = [int(i) for i in unique_ids]
+    send_local, send_slot, counts = [], [], []
+    for g in range(G):
+        mine = [u for u, i in enumerate(unique_ids) if i % G == g]
+        counts.append(len(mine))
+        send_slot += mine
+        send_local += [unique_ids[u] // G for u in mine]
+    return {"send_local": np.asarray(send_local, dtype=np.int32), "send_slot": np.asarray(send_slot, dtype=np.int32),
+            "send_counts": np.asarray(counts, dtype=np.int32)}
+
+
+def shard_owner_gradient(per_rank, V: int, G: int, g: int):
+    """What owner g holds after the gradient exchange: for each of its rows that any rank
+    touched (ascending local index), the sum over ranks of that rank's table-gradient row.
+    per_rank: list of (unique_ids, dE_rows) as returned by backward()."""
+    F = np.asarray(per_rank[0][1]).shape[1]
+    total = np.zeros((V, F), dtype=np.float64)
+    touched = np.zeros(V, dtype=bool)
+    for unique_ids, rows in per_rank:
+        total += dE_dense(unique_ids, rows, V)
+        touched[np.asarray(unique_ids, dtype=np.int64)] = True
+    ids = np.array([i for i in range(V) if touched[i] and i % G == g], dtype=np.int64)
+    return (ids // G).astype(np.int32), total[ids]
 
 
 def ffn_macs_per_token(d: int, d_ff: int, stem: bool) -> int:

@@ -32,6 +32,7 @@ EXPORTS = (
     "stem_dagger_forward", "stem_dagger_backward", "stem_prefetch_rows", "stem_prefetch_rows_hot", "stem_lfu_workspace_bytes", "stem_lfu_touch", "stem_lfu_refresh", "stem_writeback_rows", "stem_writeback_rows_dma", "stem_gemm_bf16", "stem_step_arena_bytes",
     "stem_ffn_step_host", "stem_ffn_step_host_flush", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
     "stem_dedup_ids_static", "stem_dedup_static_max_tokens",
+    "stem_shard_route_workspace_bytes", "stem_shard_route", "stem_reduce_rows", "stem_gather_rows",
 )
 
 
@@ -84,6 +85,10 @@ def lib() -> ctypes.CDLL:
             "stem_dedup_static_max_tokens": [],
             "stem_ffn_step_host": [shp] + [vp] * 15 + [sz, vp],
             "stem_ffn_step_host_flush": [vp],
+            "stem_shard_route_workspace_bytes": [i32, i32, ctypes.POINTER(sz)],
+            "stem_shard_route": [i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
+            "stem_reduce_rows": [shp, vp, vp, vp, vp, vp, vp, sz, vp],
+            "stem_gather_rows": [shp, vp, vp, vp, vp, vp, vp],
             "stem_profile_enable": [ctypes.c_int],
             "stem_profile_count": [],
             "stem_profile_get": [ctypes.c_int, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float)],
@@ -240,6 +245,29 @@ def stem_ffn_step_host(shape, host_x, host_ids, host_dy, W_gate, E, W_down, host
 def stem_ffn_step_host_flush(stream=None) -> None:
     """Make `stream` wait for the output copies of every stem_ffn_step_host call so far."""
     _check(lib().stem_ffn_step_host_flush(_stream(stream)), "stem_ffn_step_host_flush")
+
+
+def stem_shard_route_workspace_bytes(n_max: int, G: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().stem_shard_route_workspace_bytes(n_max, G, ctypes.byref(out)), "stem_shard_route_workspace_bytes")
+    return out.value
+
+
+def stem_shard_route(n_max: int, T: int, G: int, unique_ids, n_unique, inverse, send_local, send_slot, send_counts,
+                     token_slot, route_ws, stream=None) -> None:
+    _check(lib().stem_shard_route(n_max, T, G, _p(unique_ids), _p(n_unique), _p(inverse), _p(send_local),
+                                  _p(send_slot), _p(send_counts), _p(token_slot), _p(route_ws), route_ws.numel(),
+                                  _stream(stream)), "stem_shard_route")
+
+
+def stem_gather_rows(shape, ids, n_ids, table, out, ws=None, stream=None) -> None:
+    _check(lib().stem_gather_rows(ctypes.byref(shape), _p(ids), _p(n_ids), _p(table), _p(out), _p(ws), _stream(stream)),
+           "stem_gather_rows")
+
+
+def stem_reduce_rows(shape, rows_in, perm, seg_offsets, n_unique, rows_out, ws, stream=None) -> None:
+    _check(lib().stem_reduce_rows(ctypes.byref(shape), _p(rows_in), _p(perm), _p(seg_offsets), _p(n_unique),
+                                  _p(rows_out), _p(ws), ws.numel(), _stream(stream)), "stem_reduce_rows")
 
 
 def stem_launch_count() -> int:

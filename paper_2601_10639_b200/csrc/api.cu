@@ -327,6 +327,62 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
   return STEM_OK;
 }
 
+// ---- table sharded over GPUs ---------------------------------------------------------------
+int stem_shard_route_workspace_bytes(int32_t n_max, int32_t G, size_t* bytes) {
+  if (!bytes || n_max < 0 || G < 1 || G > 1024) return STEM_ERR_INVALID_ARG;
+  if (n_max > (1 << 22)) return STEM_ERR_UNSUPPORTED_SHAPE;
+  *bytes = shard_route_workspace_bytes(n_max, G);
+  return STEM_OK;
+}
+
+int stem_shard_route(int32_t n_max, int32_t T, int32_t G, const int32_t* unique_ids, const int32_t* n_unique,
+                     const int32_t* inverse, int32_t* send_local, int32_t* send_slot, int32_t* send_counts,
+                     int32_t* token_slot, void* route_ws, size_t route_ws_bytes, void* stream) {
+  if (n_max < 0 || T < 0 || G < 1 || G > 1024) return STEM_ERR_INVALID_ARG;
+  if (n_max > (1 << 22) || T > (1 << 22)) return STEM_ERR_UNSUPPORTED_SHAPE;
+  if (!send_counts || !route_ws || !aligned16(route_ws)) return STEM_ERR_INVALID_ARG;
+  if (n_max > 0 && (!unique_ids || !n_unique || !send_local || !send_slot)) return STEM_ERR_INVALID_ARG;
+  if (token_slot && T > 0 && !inverse) return STEM_ERR_INVALID_ARG;
+  if (route_ws_bytes < shard_route_workspace_bytes(n_max, G)) return STEM_ERR_WORKSPACE_TOO_SMALL;
+  ProfScope prof("shard_route", static_cast<cudaStream_t>(stream));
+  // no status word: the sort keys are made here and cannot be out of range
+  cudaError_t e = launch_shard_route(n_max, T, G, unique_ids, n_unique, inverse, send_local, send_slot, send_counts,
+                                     token_slot, route_ws, nullptr, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
+int stem_gather_rows(const stem_shape_t* shape, const int32_t* ids, const int32_t* n_ids, const void* table,
+                     void* out, void* ws, void* stream) {
+  if (int rc = check_shape(shape)) return rc;
+  if (shape->T == 0) return STEM_OK;
+  if (!ids || !n_ids || !table || !out || !aligned16(table) || !aligned16(out)) return STEM_ERR_INVALID_ARG;
+  const void* src = nullptr;
+  bool on_host = false;
+  if (int rc = pinned_or_device(table, &src, &on_host)) return rc;
+  const size_t row_bytes = static_cast<size_t>(shape->d_ff) * elem_bytes(shape->dtype);
+  ProfScope prof("gather_rows", static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_gather_rows(shape->T, shape->V, row_bytes, ids, n_ids, src, on_host, nullptr, nullptr, out,
+                                     ws ? status_of(ws) : nullptr, nullptr, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
+int stem_reduce_rows(const stem_shape_t* shape, const void* rows_in, const int32_t* perm,
+                     const int32_t* seg_offsets, const int32_t* n_unique, void* rows_out, void* ws,
+                     size_t ws_bytes, void* stream) {
+  if (int rc = check_shape(shape)) return rc;
+  if (!ws || !aligned16(ws)) return STEM_ERR_INVALID_ARG;
+  if (shape->T == 0) return STEM_OK;
+  if (!rows_in || !perm || !seg_offsets || !n_unique || !rows_out || !aligned16(rows_in) || !aligned16(rows_out))
+    return STEM_ERR_INVALID_ARG;
+  const WsLayout w = ws_layout(shape);
+  if (ws_bytes < w.total) return STEM_ERR_WORKSPACE_TOO_SMALL;
+  ProfScope prof("reduce_rows", static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_segreduce(shape->T, shape->d_ff, shape->grad_dtype, shape->grad_dtype, rows_in, perm,
+                                   seg_offsets, n_unique, rows_out, static_cast<char*>(ws) + w.part_off,
+                                   static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
 // ---- STEM-dagger: the up-projection is kept and the table row is added to its output -------
 int stem_dagger_forward(const stem_shape_t* shape, const void* x, const int32_t* ids, const void* W_gate,
                         const void* W_up, const void* E, const void* W_down, void* y, void* G_save, void* H_save,

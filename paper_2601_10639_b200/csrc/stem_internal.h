@@ -113,6 +113,13 @@ cudaError_t launch_lfu_refresh(int V, int K, size_t row_bytes, const int32_t* fr
                                int32_t* hot_ids, void* hot_rows, const void* table, int32_t* n_installed,
                                void* scratch, cudaStream_t stream);
 
+// ---- table sharded over GPUs: requests of the row exchange ---------------------------------
+size_t shard_route_workspace_bytes(int n_max, int G);
+cudaError_t launch_shard_route(int n_max, int T, int G, const int32_t* unique_ids, const int32_t* n_unique,
+                               const int32_t* inverse, int32_t* send_local, int32_t* send_slot,
+                               int32_t* send_counts, int32_t* token_slot, void* scratch, int32_t* status,
+                               cudaStream_t stream);
+
 int device_sm_count();
 
 // Function attributes (shared-memory size, preferred split) are per device: `done` is a

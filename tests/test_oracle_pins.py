@@ -380,3 +380,47 @@ def test_dagger_reduces_to_dense_swiglu_autograd_and_to_the_layer():
     y_dense = (O.silu(c["x"] @ c["W_gate"].T) * (c["x"] @ W_up.T)) @ c["W_down"].T
     np.testing.assert_allclose(O.dagger_forward(c["x"], c["ids"], c["W_gate"], W_up, np.zeros_like(c["E"]), c["W_down"]),
                                y_dense, **kw)
+
+
+@pytest.mark.parametrize("G", [1, 2, 3, 8])
+def test_shard_route_is_a_partition_that_reconstructs_every_id(G):
+    """Routing pin: every distinct id is requested exactly once, from the rank its id mod G
+    names, by the local index that gives the id back; groups are in owner order, ascending
+    inside; G = 1 is the identity."""
+    rng = np.random.default_rng(5 + G)
+    unique_ids = np.sort(rng.choice(1000, size=137, replace=False)).astype(np.int32)
+    r = O.shard_route(unique_ids, G)
+    assert int(r["send_counts"].sum()) == len(unique_ids) and len(r["send_counts"]) == G
+    assert sorted(r["send_slot"].tolist()) == list(range(len(unique_ids)))        # a permutation
+    owner = np.repeat(np.arange(G), r["send_counts"])
+    assert np.array_equal(r["send_local"].astype(np.int64) * G + owner, unique_ids[r["send_slot"]])
+    for g in range(G):
+        grp = unique_ids[r["send_slot"][owner == g]]
+        assert np.all(grp % G == g) and np.all(np.diff(grp) > 0)
+    if G == 1:
+        assert np.array_equal(r["send_local"], unique_ids) and np.array_equal(r["send_slot"], np.arange(137))
+
+
+def test_owner_gradient_is_the_table_gradient_of_the_concatenated_batches():
+    """The loss is a sum over positions, so the owners' sums over ranks must equal the table
+    gradient of all ranks' positions taken as one batch, restricted to each owner's rows."""
+    rng = np.random.default_rng(11)
+    T, d, F, V, G = 40, 8, 12, 30, 3
+    W_gate, W_down, E = rng.normal(size=(F, d)), rng.normal(size=(d, F)), rng.normal(size=(V, F))
+    xs = [rng.normal(size=(T, d)) for _ in range(G)]
+    dys = [rng.normal(size=(T, d)) for _ in range(G)]
+    idss = [rng.integers(0, V, size=T).astype(np.int32) for _ in range(G)]
+    per_rank = []
+    for r in range(G):
+        bw = O.backward(dys[r], xs[r], idss[r], W_gate, E, W_down)
+        per_rank.append((bw["unique_ids"], bw["dE_rows"]))
+    whole = O.backward(np.concatenate(dys), np.concatenate(xs), np.concatenate(idss), W_gate, E, W_down)
+    dense = O.dE_dense(whole["unique_ids"], whole["dE_rows"], V)
+    seen = set()
+    for g in range(G):
+        local, rows = O.shard_owner_gradient(per_rank, V, G, g)
+        ids = local.astype(np.int64) * G + g
+        assert np.all(np.diff(ids) > 0)
+        np.testing.assert_allclose(rows, dense[ids], rtol=1e-12, atol=1e-12)
+        seen |= set(ids.tolist())
+    assert seen == set(np.asarray(whole["unique_ids"]).tolist())
