@@ -527,6 +527,81 @@ def run_unique_growth(args):
                       "config": {"workload": "unique_growth", "V": w.V, "d_ff": w.d_ff, "ids": w.id_dist}, "rows": rows}))
 
 
+def run_sharded(args, w):
+    """The layer with its table sharded over G ranks (paper Section 3.4, "parallel embeddings"),
+    as G virtual ranks stepped in lock step on one GPU: the device time each step of a rank's
+    path takes, and the bytes its exchanges would carry.  The exchange itself is slice copies
+    here; its time over NVLink is projected, not measured."""
+    import torch
+    from paper_2601_10639_b200 import binding as B
+    from paper_2601_10639_b200 import runner, sharded
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    B.lib()
+    G = args.shard_ranks
+    dt = torch.bfloat16
+    T, d, F, V = (args.tokens or w.T), w.d_model, w.d_ff, w.V
+    gen = torch.Generator(device=dev).manual_seed(args.seed)
+    shape = B.make_shape(T, d, F, V, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    W_gate = (torch.randn(F, d, generator=gen, device=dev) * d ** -0.5).to(dt)
+    W_down = (torch.randn(d, F, generator=gen, device=dev) * F ** -0.5).to(dt)
+    E = torch.empty(V, F, device=dev, dtype=dt)
+    for r0 in range(0, V, 4096):
+        r1 = min(V, r0 + 4096)
+        E[r0:r1] = (torch.randn(r1 - r0, F, generator=gen, device=dev) * 0.02).to(dt)
+    ranks = [sharded.ShardedRank(r, G, shape, E[r::G].contiguous(), W_gate, W_down, device=dev) for r in range(G)]
+    xs = [torch.randn(T, d, generator=gen, device=dev).to(dt) for _ in range(G)]
+    dys = [torch.randn(T, d, generator=gen, device=dev).to(dt) for _ in range(G)]
+    idss = [torch.from_numpy(synth.token_ids(rank_seed(args.seed, r), T, V, w.id_dist)).to(dev) for r in range(G)]
+    ex = sharded.LocalExchange(G)
+    steps = min(args.steps, 20)
+    for _ in range(3):
+        sharded.step_local(ranks, ex, xs, idss, dys)
+    torch.cuda.synchronize()
+    launches0 = B.stem_launch_count()
+    events = []
+
+    def timed(name, fn):      # CUDA events around one rank's phase: the exchange's copies stay outside
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        out = fn()
+        e1.record()
+        events.append((name, e0, e1))
+        return out
+
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        owned = sharded.step_local(ranks, ex, xs, idss, dys, timed)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    assert all(r.status() == B.OK for r in ranks)
+    per_rank_step = {}
+    for name, e0, e1 in events:
+        per_rank_step[name] = per_rank_step.get(name, 0.0) + e0.elapsed_time(e1) / (steps * G)
+    # route = dedup + requests (+ the count read-back); serve = the owner's gather; layer = forward,
+    # backward and the gradient rows put in request order; reduce = the owner's dedup + per-row sums
+    layer = per_rank_step["layer"]
+    extra = per_rank_step["route"] + per_rank_step["serve"] + per_rank_step["reduce"]
+    n_u = sum(r.h_send_counts[g] for r in ranks for g in range(G)) / G
+    remote = sum(r.h_send_counts[g] for r in ranks for g in range(G) if g != r.rank) / G
+    fwd_bytes, bwd_bytes = remote * F * 2, remote * F * 4
+    nvlink_gbs = 770.0
+    print(json.dumps({
+        "metric": "STEM-FFN fwd+bwd with the table sharded over G ranks: device time per rank per step",
+        "value": T / ((layer + extra) * 1e-3), "unit": "tokens/s per rank (exchange time excluded)",
+        "n_gpus": 1, "virtual_ranks": G, "steps": steps, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "tokens_per_rank": T, "d_model": d, "d_ff": F, "V": V, "ids": w.id_dist,
+                   "rows_by": "id mod G", "exchange": "in-process slice copies (one GPU); NVLink time projected"},
+        "ms_per_rank_step": {"layer": layer, "route_serve_reduce": extra, **per_rank_step},
+        "distinct_rows_per_rank": n_u, "rows_from_other_ranks": remote,
+        "exchange_bytes_per_rank": {"rows_in": fwd_bytes, "grad_rows_out_fp32": bwd_bytes},
+        "projected_exchange_ms_at_770GBs": {"rows_in": fwd_bytes / nvlink_gbs / 1e6, "grad_rows_out": bwd_bytes / nvlink_gbs / 1e6},
+        "owner_rows_reduced": [int(o[1].item()) for o in owned],
+        "gpu_launches": B.stem_launch_count() - launches0, "wall_ms_per_step_all_ranks": wall / steps * 1e3,
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -548,6 +623,8 @@ def main():
     ap.add_argument("--no-profile", action="store_true",
                     help="do not record per-step events inside the timed region (checks what they cost)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
+    ap.add_argument("--shard-ranks", type=int, default=0,
+                    help="G > 0: the table sharded over G virtual ranks on one GPU (per-rank device times)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.warmup < 3:
@@ -560,6 +637,11 @@ def main():
         run_unique_growth(args)
         return
 
+    if args.shard_ranks > 0:
+        if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+            raise SystemExit("--shard-ranks steps virtual ranks on one GPU")
+        run_sharded(args, w)
+        return
     if w.host_tables:
         if int(os.environ.get("WORLD_SIZE", "1")) > 1:
             raise SystemExit("the host-table workload is a one-GPU measurement")

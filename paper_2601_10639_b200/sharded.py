@@ -142,28 +142,46 @@ class ShardedRank:
         return self.grad_send[:n_u]
 
     # -- D: owner side of the gradient exchange ----------------------------------------------
-    def phase_reduce(self, recv_rows: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
-        """Returns (local row indices ascending, summed gradient rows) for this rank's shard."""
+    def _owner_buffers(self, n: int, dtype):
+        """Index arrays, output rows and workspace of the owner's reduce, kept between steps and
+        regrown (with headroom) when a step brings more rows than any before."""
+        ob = getattr(self, "_ob", None)
+        if ob is None or ob["cap"] < n or ob["rows"].dtype != dtype:
+            s, dev = self.shape, self.device
+            cap = max(int(n * 1.25), 16)
+            rows_local = max(self.shard.shape[0], 1)
+            R = max(min(cap, rows_local), 1)
+            shp = B.make_shape(cap, s.d_model, s.d_ff, rows_local, s.dtype, s.grad_dtype, 0)
+            ws = torch.empty(max(B.stem_workspace_bytes(shp), 256), dtype=torch.uint8, device=dev)
+            B.stem_init_workspace(ws)
+            ob = {"cap": cap, "ws": ws, "uniq": torch.empty(R, dtype=torch.int32, device=dev),
+                  "n_u": torch.zeros(1, dtype=torch.int32, device=dev),
+                  "inv": torch.empty(cap, dtype=torch.int32, device=dev),
+                  "perm": torch.empty(cap, dtype=torch.int32, device=dev),
+                  "seg": torch.empty(R + 1, dtype=torch.int32, device=dev),
+                  "rows": torch.empty(R, s.d_ff, dtype=dtype, device=dev)}
+            self._ob = ob
+        return ob
+
+    def phase_reduce(self, recv_rows: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+        """Returns (local row indices ascending, their count (device scalar), summed gradient rows)
+        for this rank's shard; entries past the count are undefined.  No host synchronisation."""
         n = int(self.recv_local.numel())
         s = self.shape
+        ob = self._owner_buffers(n, recv_rows.dtype)
         if n == 0:
-            return self.recv_local[:0], recv_rows[:0]
-        rows_local = self.shard.shape[0]
-        oshape = B.make_shape(n, s.d_model, s.d_ff, rows_local, s.dtype, s.grad_dtype, 0)
-        R = max(min(n, rows_local), 1)
-        ws = torch.empty(max(B.stem_workspace_bytes(oshape), 256), dtype=torch.uint8, device=self.device)
-        B.stem_init_workspace(ws)
-        uniq = torch.empty(R, dtype=torch.int32, device=self.device)
-        n_u = torch.zeros(1, dtype=torch.int32, device=self.device)
-        inv = torch.empty(n, dtype=torch.int32, device=self.device)
-        perm = torch.empty(n, dtype=torch.int32, device=self.device)
-        seg = torch.empty(R + 1, dtype=torch.int32, device=self.device)
-        B.stem_dedup_ids(oshape, self.recv_local, uniq, n_u, inv, perm, seg, ws)
-        out = torch.empty(R, s.d_ff, dtype=recv_rows.dtype, device=self.device)
-        B.stem_reduce_rows(oshape, recv_rows.contiguous(), perm, seg, n_u, out, ws)
-        k = int(n_u.item())
-        self.owner_status = B.stem_query_status(ws)
-        return uniq[:k], out[:k]
+            ob["n_u"].zero_()
+            return ob["uniq"], ob["n_u"], ob["rows"]
+        oshape = B.make_shape(n, s.d_model, s.d_ff, max(self.shard.shape[0], 1), s.dtype, s.grad_dtype, 0)
+        B.stem_dedup_ids(oshape, self.recv_local, ob["uniq"], ob["n_u"], ob["inv"], ob["perm"], ob["seg"], ob["ws"])
+        B.stem_reduce_rows(oshape, recv_rows.contiguous(), ob["perm"], ob["seg"], ob["n_u"], ob["rows"], ob["ws"])
+        return ob["uniq"], ob["n_u"], ob["rows"]
+
+    def status(self) -> int:
+        """First device-side error of either role (synchronises)."""
+        st = self.layer.status()
+        ob = getattr(self, "_ob", None)
+        return st if st != B.OK or ob is None else B.stem_query_status(ob["ws"])
 
     # -- one step, one process per GPU ---------------------------------------------------------
     def step_dist(self, ex: DistExchange, x, ids, dy):
@@ -178,14 +196,16 @@ class ShardedRank:
         return self.phase_reduce(recv_grads)
 
 
-def step_local(ranks: List[ShardedRank], ex: LocalExchange, xs, idss, dys):
-    """One step of G virtual ranks in lock step (single process, single GPU)."""
+def step_local(ranks: List[ShardedRank], ex: LocalExchange, xs, idss, dys, timed=None):
+    """One step of G virtual ranks in lock step (single process, single GPU).  `timed(name, fn)`
+    may wrap each rank's phase (the benchmark brackets them with CUDA events)."""
     G = ex.G
-    send_counts = [ranks[r].phase_route(xs[r], idss[r], dys[r]) for r in range(G)]
+    run = timed or (lambda name, fn: fn())
+    send_counts = [run("route", lambda r=r: ranks[r].phase_route(xs[r], idss[r], dys[r])) for r in range(G)]
     recv_counts = ex.counts_all(send_counts)
     recv_local = ex.rows_all([ranks[r].send_local[:sum(send_counts[r])] for r in range(G)], send_counts)
-    served = [ranks[r].phase_serve(recv_local[r], recv_counts[r]) for r in range(G)]
+    served = [run("serve", lambda r=r: ranks[r].phase_serve(recv_local[r], recv_counts[r])) for r in range(G)]
     rows = ex.rows_all(served, recv_counts)
-    grads = [ranks[r].phase_layer(rows[r]) for r in range(G)]
+    grads = [run("layer", lambda r=r: ranks[r].phase_layer(rows[r])) for r in range(G)]
     recv_grads = ex.rows_all(grads, send_counts)
-    return [ranks[r].phase_reduce(recv_grads[r]) for r in range(G)]
+    return [run("reduce", lambda r=r: ranks[r].phase_reduce(recv_grads[r])) for r in range(G)]

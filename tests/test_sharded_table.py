@@ -48,7 +48,7 @@ def test_sharded_step_matches_the_checker(G, T, d, F, V, dist_name, grad):
     torch.cuda.synchronize()
     per_rank_ref = []
     for r in range(G):
-        assert ranks[r].layer.status() == B.OK
+        assert ranks[r].status() == B.OK
         y_ref = O.forward(per[r]["x"], per[r]["ids"], base["W_gate"], base["E"], base["W_down"])
         bw = O.backward(per[r]["dy"], per[r]["x"], per[r]["ids"], base["W_gate"], base["E"], base["W_down"])
         per_rank_ref.append((bw["unique_ids"], bw["dE_rows"]))
@@ -65,10 +65,10 @@ def test_sharded_step_matches_the_checker(G, T, d, F, V, dist_name, grad):
         assert np.array_equal(ranks[r].send_slot[:n_u].cpu().numpy(), route["send_slot"])
     for g in range(G):
         local_ref, rows_ref = O.shard_owner_gradient(per_rank_ref, V, G, g)
-        local, rows = owned[g]
-        assert np.array_equal(local.cpu().numpy(), local_ref)
-        assert O.scaled_max_err(_np(rows), rows_ref) <= TOL_BF16
-        assert getattr(ranks[g], "owner_status", B.OK) == B.OK
+        local, count, rows = owned[g]
+        k = int(count.item())
+        assert np.array_equal(local[:k].cpu().numpy(), local_ref)
+        assert O.scaled_max_err(_np(rows[:k]), rows_ref) <= TOL_BF16
 
 
 @pytest.mark.gpu
