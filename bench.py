@@ -477,6 +477,49 @@ def run_decode(args, w):
     ev1.record(stream)
     torch.cuda.synchronize()
     res_ms = ev0.elapsed_time(ev1) / 200
+
+    # The same two loops replayed from CUDA graphs: a decode step is a handful of short launches,
+    # so how fast the host can issue them is part of the eager figures above.  The step's ids are
+    # copied into a fixed buffer before each replay; the cache refresh stays outside the graph.
+    def replay_ms(body, n, before=None):
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(3):
+                body()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            body()
+        for i in range(10):
+            if before:
+                before(i)
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            if before:
+                before(i)
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    ids_now = all_ids[:Bt].clone()
+    res_graph_ms = replay_ms(lambda: B.stem_ffn_forward(shape, x, ids_now, W_gate, dev_table, W_down, b["y"], None, None,
+                                                       b["ws"]), 200)
+
+    def graph_body():
+        B.stem_lfu_touch(Bt, V, ids_now, freq, hot_slot, stats)
+        B.stem_dedup_ids(shape, ids_now, b["unique_ids"], b["n_unique"], b["inverse"], b["perm"], b["seg_offsets"], b["ws"])
+        B.stem_prefetch_rows_hot(shape, b["unique_ids"], b["n_unique"], table, hot_rows, hot_slot, cache, rows, b["ws"])
+        B.stem_ffn_forward(cshape, x, b["inverse"], W_gate, cache, W_down, b["y"], None, None, b["ws"])
+
+    half = steps // 2
+    step_graph_ms = replay_ms(graph_body, steps - half, lambda i: ids_now.copy_(all_ids[(half + i) * Bt:(half + i + 1) * Bt]))
+    assert st.status() == B.OK
     best = min(out.values(), key=lambda r: r["ms_per_step"])
     peaks = load_peaks()
     wbytes = 2 * d * F * 2
@@ -488,6 +531,9 @@ def run_decode(args, w):
         "config": {"workload": w.name, "tokens_per_step": Bt, "d_model": d, "d_ff": F, "V": V, "ids": w.id_dist,
                    "paper_hit_rate": "> 80 % (Section 3.4, hardware and cache size not stated)"},
         "modes": out, "device_table_forward_ms": res_ms,
+        "cuda_graph": {"device_table_forward_ms": res_graph_ms, "step_ms": step_graph_ms, "hot_rows": args.hot_rows[-1],
+                       "tokens_per_s": Bt / (step_graph_ms * 1e-3),
+                       "note": "the step (count, dedup, gather, forward) captured once and replayed; ids copied in before each replay"},
         "roofline": {"bound": "hbm", "achieved": wbytes / (res_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": wbytes / (res_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
                      "kernel": "forward with a device table (both weight matrices read once per step: 2 d d_ff elements, Table 1)",
