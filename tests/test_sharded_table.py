@@ -26,6 +26,12 @@ def _np(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 @pytest.mark.gpu
 @pytest.mark.parametrize("G,T,d,F,V,dist_name,grad", [
     (2, 300, 264, 520, 1000, "zipf", B.DTYPE_FP32),
@@ -72,6 +78,32 @@ def test_sharded_step_matches_the_checker(G, T, d, F, V, dist_name, grad):
 
 
 @pytest.mark.gpu
+def test_one_rank_step_over_nccl():
+    """The torch.distributed exchange on the device (NCCL, a group of one: every all-to-all is a
+    copy to self), driving the same phases as the virtual ranks."""
+    T, d, F, V = 300, 128, 264, 500
+    w = synth.Workload("t", T, d, F, V, "bf16", "zipf")
+    inp = synth.make_inputs(w, seed=310)
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{_free_port()}", rank=0, world_size=1,
+                            device_id=torch.device("cuda", 0))
+    try:
+        E = runner.to_device(inp["E"], B.DTYPE_BF16)
+        rk = sharded.ShardedRank(0, 1, B.make_shape(T, d, F, V, B.DTYPE_BF16, B.DTYPE_FP32, 0), E,
+                                 runner.to_device(inp["W_gate"], B.DTYPE_BF16), runner.to_device(inp["W_down"], B.DTYPE_BF16))
+        local, count, rows = rk.step_dist(sharded.DistExchange(), runner.to_device(inp["x"], B.DTYPE_BF16),
+                                          runner.to_device(inp["ids"], B.DTYPE_BF16), runner.to_device(inp["dy"], B.DTYPE_BF16))
+        torch.cuda.synchronize()
+        assert rk.status() == B.OK
+    finally:
+        dist.destroy_process_group()
+    bw = O.backward(inp["dy"], inp["x"], inp["ids"], inp["W_gate"], inp["E"], inp["W_down"])
+    k = int(count.item())
+    assert np.array_equal(local[:k].cpu().numpy(), bw["unique_ids"])        # G = 1: local index = id
+    assert O.scaled_max_err(_np(rows[:k]), bw["dE_rows"]) <= TOL_BF16
+    assert O.scaled_max_err(_np(rk.layer.bufs["dx"]), bw["dx"]) <= TOL_BF16
+
+
+@pytest.mark.gpu
 def test_reduce_rows_and_gather_rows_alone():
     """The two calls of the owner's side on their own: repeated ids in the gather, the reduce
     against per-index sums (fp32 rows are added in a fixed order, so twice gives the same bits)."""
@@ -106,12 +138,6 @@ def test_reduce_rows_and_gather_rows_alone():
 
 
 # ---- the exchange itself, as two gloo ranks on the CPU ----------------------------------------
-def _free_port() -> int:
-    with socket.socket() as s:
-        s.bind(("127.0.0.1", 0))
-        return s.getsockname()[1]
-
-
 def _case(G):
     rng = np.random.default_rng(17)
     counts = [[int(rng.integers(0, 5)) for _ in range(G)] for _ in range(G)]       # counts[src][dst]
