@@ -148,7 +148,7 @@ int stem_ffn_forward(const stem_shape_t* shape, const void* x, const int32_t* id
 
 /*
  * Backward.  The paper states no formulas (training is implied: Table 1 notes, Section
- * 3.3); these are the chain rule of the layer equation for L = sum dy (.) y:
+ * 3.4); these are the chain rule of the layer equation for L = sum dy (.) y:
  *   dH = dy W_down;  dU = dH (.) SiLU(G);  dG = dH (.) E[ids] (.) SiLU'(G)
  *   dW_down = dy^T H;  dW_gate = dG^T x;  dx = dG W_gate
  *   dE_rows[r] = sum of dU[t] over the positions t with ids[t] == unique_ids[r]
@@ -157,7 +157,8 @@ int stem_ffn_forward(const stem_shape_t* shape, const void* x, const int32_t* id
  * unique_ids: from stem_dedup_ids on the same ids.  dE_rows [min(T,V), d_ff]
  * (grad_dtype): rows >= n_u are left untouched; ids absent from the call have no row
  * (their gradient is zero).  dW_gate, dW_down in grad_dtype; dx in dtype.  Any of dx,
- * dW_gate, dW_down, dE_rows may be NULL to skip that output.
+ * dW_gate, dW_down, dE_rows may be NULL to skip that output.  With STEM_FLAG_ACCUM_GRADS in
+ * shape->flags, dW_gate and dW_down are added to instead of overwritten.
  */
 int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, const int32_t* ids,
                       const void* W_gate, const void* E, const void* W_down, const void* G_save,
