@@ -207,6 +207,24 @@ def test_weight_gradients_accumulate_over_micro_batches(flags, T, d, F, grad):
     assert all(v <= TOL_BF16 for v in errs.values()), errs
 
 
+def test_randomized_shapes_layouts_and_gradient_types():
+    """Forty seeded draws of (T, d_model, d_ff, V, id mix, CTA pairs or single CTAs, gradient type):
+    ragged tiles in every dimension, tables of one row, batches of one position."""
+    rng = np.random.default_rng(424242)
+    for case in range(40):
+        T = int(rng.choice([1, 2, 7, 31, 64, 127, 129, 255, 257, 300, 511, 640, 1000, 1025, 2049, 3000]))
+        d, F = int(rng.integers(1, 140)) * 8, int(rng.integers(1, 160)) * 8
+        V = int(rng.choice([1, 2, 5, 37, 300, 4096, 32000]))
+        dist = str(rng.choice(["zipf", "uniform", "same"]))
+        flags = int(rng.choice([0, B.FLAG_SINGLE_CTA]))
+        grad = int(rng.choice([B.DTYPE_FP32, B.DTYPE_BF16]))
+        w = synth.Workload("t", T, d, F, V, "bf16", dist)
+        try:
+            _full_parity(w, synth.make_inputs(w, seed=7000 + case), B.DTYPE_BF16, TOL_BF16, flags, grad_dtype=grad)
+        except AssertionError as e:
+            raise AssertionError(f"case {case}: T={T} d={d} F={F} V={V} {dist} flags={flags} grad={grad}: {e}") from e
+
+
 def test_backward_is_bitwise_reproducible():
     w = synth.Workload("t", 2048, 256, 1024, 500, "bf16", "zipf")
     st = runner.state_from_numpy(synth.make_inputs(w, seed=79), B.DTYPE_BF16, w.V)
