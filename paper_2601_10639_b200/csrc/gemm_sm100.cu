@@ -473,7 +473,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // Fix-up for the tail tiles: output tile = sum of its pieces in ascending k order (piece ik of
-// tail tile j is slot ik * tail + j).  One CTA per (tail tile, 32-row band).
+// tail tile j is slot ik * tail + j).  One CTA per (tail tile, kFixRows-row band); a thread
+// requests its element of every piece before it adds the first, so the launch is bound by
+// bandwidth (the partial tiles mostly still sit in L2), not by a chain of load latencies.
+constexpr int kMaxSplit = 8;   // most pieces a tail tile is cut into
+constexpr int kFixRows = 8;    // rows of a tile per fix-up CTA
 template <int BN, int CTAS>
 __global__ void __launch_bounds__(256)
 tail_fixup_kernel(int M, int N, int dp_tiles, int tail, int split, int tiles_m, int tiles_n, int group_m,
@@ -483,16 +487,23 @@ tail_fixup_kernel(int M, int N, int dp_tiles, int tail, int split, int tiles_m, 
   ptx::grid_launch_dependents();
   const int j = blockIdx.x;
   const TileCoord tc = tile_coord(dp_tiles + j, tiles_m, tiles_n, group_m);
-  const int r0 = blockIdx.y * 32;
-  for (int e = threadIdx.x; e < 32 * (BN / 4); e += 256) {
+  const int r0 = blockIdx.y * kFixRows;
+  for (int e = threadIdx.x; e < kFixRows * (BN / 4); e += 256) {
     const int r = r0 + e / (BN / 4), c = (e % (BN / 4)) * 4;
     const int m = tc.m_blk * TM + r, nn = tc.n_blk * BN + c;
     if (m >= M || nn >= N) continue;
+    float4 v[kMaxSplit];
+#pragma unroll
+    for (int ik = 0; ik < kMaxSplit; ++ik) {
+      if (ik < split) {
+        const size_t slot = static_cast<size_t>(ik) * tail + j;
+        v[ik] = __ldcg(reinterpret_cast<const float4*>(partial + (slot * TM + r) * BN + c));
+      }
+    }
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int ik = 0; ik < split; ++ik) {
-      const size_t slot = static_cast<size_t>(ik) * tail + j;
-      const float4 v = *reinterpret_cast<const float4*>(partial + (slot * TM + r) * BN + c);
-      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+#pragma unroll
+    for (int ik = 0; ik < kMaxSplit; ++ik) {
+      if (ik < split) { acc.x += v[ik].x; acc.y += v[ik].y; acc.z += v[ik].z; acc.w += v[ik].w; }
     }
     const size_t o = static_cast<size_t>(m) * N + nn;   // N is a multiple of 8: 4 columns never straddle the edge
     if (out_fp32) {
@@ -596,7 +607,7 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
   count_launches(1);
   if (e == cudaSuccess && sk_tail > 0) {
     cudaLaunchConfig_t fcfg = {};
-    fcfg.gridDim = dim3(sk_tail, BM * CTAS / 32);
+    fcfg.gridDim = dim3(sk_tail, BM * CTAS / kFixRows);
     fcfg.blockDim = dim3(256);
     fcfg.stream = stream;
     fcfg.attrs = attr + 1;
@@ -626,7 +637,7 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
     tmC1 = tmC0;
     // The last round costs ceil(tail * split / slots) / split tile times instead of one.
     // Worth it when that saves clearly more than the partial tiles and the fix-up launch
-    // cost (~25 us); a tile time is ~ 2 TM BN K flops at ~11 TFLOP/s per SM.
+    // cost (10-25 us together); a tile time is ~ 2 TM BN K flops at ~11 TFLOP/s per SM.
     constexpr int TM = BM * CTAS;
     const int units = ((M + TM - 1) / TM) * ((N + BN - 1) / BN);
     const int slots = device_sm_count() / CTAS;
@@ -637,7 +648,7 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
     if (tail > 0 && ep.sk_scratch != nullptr) {
       int best = 1;
       double best_cost = 1.0;
-      for (int sp = 2; sp <= 8; ++sp) {
+      for (int sp = 2; sp <= kMaxSplit; ++sp) {
         if (static_cast<size_t>(tail) * sp * slot_bytes > ep.sk_bytes || k_blocks / sp < 4) break;
         const double cost = static_cast<double>((tail * sp + slots - 1) / slots) / sp;
         if (cost < best_cost - 0.04) { best_cost = cost; best = sp; }
