@@ -99,6 +99,7 @@ class ShardedRank:
         self.route_ws = torch.empty(max(B.stem_shard_route_workspace_bytes(self.n_max, G), 256), dtype=torch.uint8,
                                     device=dev)
         self.grad_send = torch.empty(self.n_max, s.d_ff, dtype=torch_dtype(s.grad_dtype), device=dev)
+        self.n_recv_dev = torch.zeros(1, dtype=torch.int32, device=dev)
         self.h_send_counts: List[int] = []
         self.h_recv_counts: List[int] = []
         self.recv_local = None
@@ -122,8 +123,8 @@ class ShardedRank:
         out = torch.empty(max(n, 1), s.d_ff, dtype=self.shard.dtype, device=self.device)
         if n:
             oshape = B.make_shape(n, s.d_model, s.d_ff, self.shard.shape[0], s.dtype, s.grad_dtype, 0)
-            n_dev = torch.tensor([n], dtype=torch.int32, device=self.device)
-            B.stem_gather_rows(oshape, recv_local, n_dev, self.shard, out, self.layer.bufs["ws"])
+            self.n_recv_dev.fill_(n)          # a device scalar set from the stream: no synchronous copy
+            B.stem_gather_rows(oshape, recv_local, self.n_recv_dev, self.shard, out, self.layer.bufs["ws"])
         return out[:n]
 
     # -- C: the layer on the received rows ------------------------------------------------------
