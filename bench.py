@@ -911,6 +911,9 @@ def main():
                    "l2": "per-step working set (~2.5 GB at 1b shapes) exceeds the 126 MB L2; no flush"},
         "gpu_launches": int(launches),
         "tflops_step": flops_step / (ms_per_step * 1e-3) / 1e12,
+        # the ids are the same for every STEM layer of a model, so their dedup can be paid once per batch
+        "value_dedup_amortised": (world * T / ((ms_per_step - kernels["dedup"]["avg_ms"]) * 1e-3)
+                                  if kernels.get("dedup") else None),
         "clocks": clock_summary,
         "roofline": roofline,
         "kernels": kernels,
