@@ -25,8 +25,9 @@ Token ids are 0-based.  There are no bias terms (Table 1 caption).
 Pins (tests/test_oracle_pins.py): dense SwiGLU on one-hot augmented input through
 torch autograd, central finite differences, brute-force per-id sums and index arrays,
 special values, permutation equivariance; the two cost-model functions against the
-percentages the paper prints (tests/golden/ffn_saving_fraction.txt).  Every function here
-has at least one pin.
+percentages the paper prints (tests/golden/ffn_saving_fraction.txt); the four error
+measures at the end (what the parity tests assert) against hand-computed cases.  Every
+function here has at least one pin.
 """
 from __future__ import annotations
 
@@ -242,9 +243,59 @@ def training_saving_fraction(d: int, d_ff: int, L: int) -> float:
 
 
 def scaled_max_err(got, ref) -> float:
-    """max |got - ref| / max |ref|  -- the error measure the parity tests use."""
+    """max |got - ref| / max |ref| over the whole tensor: the coarse measure.  Not symmetric: the
+    scale comes from `ref`.  ref identically zero (or empty): the scale is 1."""
     got, ref = _f64(got), _f64(ref)
     denom = float(np.max(np.abs(ref))) if ref.size else 1.0
     if denom == 0.0:
         denom = 1.0
     return float(np.max(np.abs(got - ref))) / denom if ref.size else 0.0
+
+
+def rel_frobenius_err(got, ref) -> float:
+    """||got - ref||_F / ||ref||_F: the error of the tensor as a whole (root of the summed
+    squares), which a handful of good large elements cannot hide.  ref identically zero (or
+    empty): the scale is 1."""
+    got, ref = _f64(got), _f64(ref)
+    if not ref.size:
+        return 0.0
+    denom = float(np.sqrt(np.sum(ref * ref)))
+    if denom == 0.0:
+        denom = 1.0
+    return float(np.sqrt(np.sum((got - ref) ** 2))) / denom
+
+
+def elementwise_pass_rate(got, ref, tol: float, per_row: bool = False) -> float:
+    """Fraction of elements with |got - ref| <= tol * (|ref| + rms(ref)).
+
+    The element's own magnitude plus the typical magnitude around it: a relative test that stays
+    defined at entries near zero.  per_row=False takes the root mean square of the whole tensor;
+    per_row=True takes it row by row (last axis), for tensors whose rows differ in scale by orders
+    of magnitude -- the table-gradient rows of a Zipfian batch, where a frequent id's row sums
+    thousands of positions and a rare id's row one, so that a rare row cannot hide behind the
+    frequent ones.  Empty input: 1.0."""
+    got, ref = _f64(got), _f64(ref)
+    if not ref.size:
+        return 1.0
+    if per_row:
+        rms = np.sqrt(np.mean(ref * ref, axis=-1, keepdims=True))
+    else:
+        rms = np.sqrt(np.mean(ref * ref))
+    ok = np.abs(got - ref) <= tol * (np.abs(ref) + rms)
+    return float(np.count_nonzero(ok)) / ref.size
+
+
+def max_row_rel_err(got, ref) -> float:
+    """max over rows r of ||got[r] - ref[r]||_2 / ||ref[r]||_2 (rows along the last axis): every row
+    judged on its own scale.  For the table-gradient rows of a Zipfian batch, where a frequent id's
+    row sums thousands of positions and a rare id's row one, this is the measure a wrong rare row
+    cannot hide from -- and, unlike a bound on single entries, it is not thrown by an entry that a
+    few large terms of opposite sign cancel to nearly zero.  A row of ref that is identically zero
+    has scale 1.  Empty input: 0."""
+    got, ref = _f64(got), _f64(ref)
+    if not ref.size:
+        return 0.0
+    num = np.sqrt(np.sum((got - ref) ** 2, axis=-1))
+    den = np.sqrt(np.sum(ref * ref, axis=-1))
+    den = np.where(den == 0.0, 1.0, den)
+    return float(np.max(num / den))

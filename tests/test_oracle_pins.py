@@ -424,3 +424,104 @@ def test_owner_gradient_is_the_table_gradient_of_the_concatenated_batches():
         np.testing.assert_allclose(rows, dense[ids], rtol=1e-12, atol=1e-12)
         seen |= set(ids.tolist())
     assert seen == set(np.asarray(whole["unique_ids"]).tolist())
+
+
+# ---------------------------------------------------------------------------------------
+# the error measures the parity tests assert: hand-computed cases (the expected numbers below are
+# worked out by hand, not by re-typing the formulas)
+# ---------------------------------------------------------------------------------------
+def test_scaled_max_err_hand_cases():
+    ref = np.array([[4.0, -2.0], [1.0, 0.5]])
+    assert O.scaled_max_err(ref, ref) == 0.0
+    # a sign flip on the -2: |(-(-2)) - (-2)| = 4, against max |ref| = 4
+    got = ref.copy(); got[0, 1] = 2.0
+    assert O.scaled_max_err(got, ref) == 1.0
+    # a slip to |got| - |ref| would call that flip exact; a mean instead of a max would give 1/4
+    # one element off by 0.25 under a maximum of 4
+    got = ref.copy(); got[1, 1] = 0.75
+    assert O.scaled_max_err(got, ref) == 0.0625
+    # the scale comes from the second argument: the measure is not symmetric
+    assert O.scaled_max_err(np.array([2.0, 0.0]), np.array([1.0, 0.0])) == 1.0
+    assert O.scaled_max_err(np.array([1.0, 0.0]), np.array([2.0, 0.0])) == 0.5
+    # the sign of the difference does not matter, the largest one decides
+    assert O.scaled_max_err(np.array([9.0, 10.0, -3.0]), np.array([10.0, 10.0, 0.0])) == 0.3
+    # ref identically zero: scale 1, the measure is the largest |got|; empty: 0
+    assert O.scaled_max_err(np.array([0.0, -0.125]), np.zeros(2)) == 0.125
+    assert O.scaled_max_err(np.zeros((0, 3)), np.zeros((0, 3))) == 0.0
+    # integers and float32 are widened, not wrapped
+    assert O.scaled_max_err(np.array([1, 2], dtype=np.int32), np.array([1.0, 4.0], dtype=np.float32)) == 0.5
+
+
+def test_rel_frobenius_err_hand_cases():
+    ref = np.array([[3.0, 0.0], [0.0, 4.0]])          # norm 5
+    assert O.rel_frobenius_err(ref, ref) == 0.0
+    got = ref + np.array([[0.0, 0.3], [0.4, 0.0]])    # difference of norm 0.5
+    assert abs(O.rel_frobenius_err(got, ref) - 0.1) < 1e-15
+    # errors on several elements add in squares: four errors of 1 -> 2, not 1 (max) and not 4 (sum)
+    assert O.rel_frobenius_err(np.ones(4) * 2.0, np.ones(4)) == 1.0     # 2 / 2
+    assert abs(O.rel_frobenius_err(np.array([1.0, 1.0, 1.0, 2.0]), np.ones(4)) - 0.5) < 1e-15
+    # scale from ref (asymmetric); ref zero -> scale 1; empty -> 0
+    assert O.rel_frobenius_err(np.array([6.0, 8.0]), np.array([3.0, 4.0])) == 1.0
+    assert O.rel_frobenius_err(np.array([3.0, 4.0]), np.array([6.0, 8.0])) == 0.5
+    assert O.rel_frobenius_err(np.array([3.0, -4.0]), np.zeros(2)) == 5.0
+    assert O.rel_frobenius_err(np.zeros(0), np.zeros(0)) == 0.0
+
+
+def test_elementwise_pass_rate_hand_cases():
+    # ref = [3, -3, 3, -3]: rms 3, so the allowance at tol 0.1 is 0.1 * (3 + 3) = 0.6 per element
+    ref = np.array([3.0, -3.0, 3.0, -3.0])
+    assert O.elementwise_pass_rate(ref, ref, 0.1) == 1.0
+    assert O.elementwise_pass_rate(ref + np.array([0.5, -0.5, 0.59, 0.0]), ref, 0.1) == 1.0
+    assert O.elementwise_pass_rate(ref + np.array([0.7, 0.0, 0.0, 0.0]), ref, 0.1) == 0.75
+    assert O.elementwise_pass_rate(ref + np.array([0.7, -0.7, 0.0, 0.0]), ref, 0.1) == 0.5
+    assert O.elementwise_pass_rate(-ref, ref, 0.1) == 0.0               # all signs flipped
+    # an element at zero is still allowed tol * rms: ref = [0, 4] has rms sqrt(8) = 2.83, allowance 0.283
+    assert O.elementwise_pass_rate(np.array([0.25, 4.0]), np.array([0.0, 4.0]), 0.1) == 1.0
+    assert O.elementwise_pass_rate(np.array([0.30, 4.0]), np.array([0.0, 4.0]), 0.1) == 0.5
+    # rows of very different scale: the small row is wrong by a factor of two.  The coarse measure
+    # and the whole-tensor allowance both let it through; the row-wise allowance does not.
+    ref2 = np.array([[100.0, -100.0], [0.01, 0.01]])
+    got2 = np.array([[100.0, -100.0], [0.02, 0.02]])
+    assert O.scaled_max_err(got2, ref2) == 1e-4
+    assert O.elementwise_pass_rate(got2, ref2, 0.02) == 1.0             # allowance 0.02 * (0.01 + 70.7)
+    assert O.elementwise_pass_rate(got2, ref2, 0.02, per_row=True) == 0.5   # allowance 0.02 * 0.02 = 4e-4 < 0.01
+    assert O.elementwise_pass_rate(ref2, ref2, 0.02, per_row=True) == 1.0
+    # row-wise on a 3-d tensor uses the last axis; empty input passes
+    assert O.elementwise_pass_rate(got2[None], ref2[None], 0.02, per_row=True) == 0.5
+    assert O.elementwise_pass_rate(np.zeros((0, 4)), np.zeros((0, 4)), 0.1, per_row=True) == 1.0
+    # ref identically zero: only exact zeros pass
+    assert O.elementwise_pass_rate(np.array([0.0, 1e-30]), np.zeros(2), 0.5) == 0.5
+
+
+def test_error_measures_catch_planted_slips():
+    """Plausible slips in the measures themselves, planted in copies, change at least one hand case."""
+    ref = np.array([[4.0, -2.0], [1.0, 0.5]])
+    flip = ref.copy(); flip[0, 1] = 2.0
+    slip_abs = lambda g, r: float(np.max(np.abs(np.abs(g) - np.abs(r)))) / float(np.max(np.abs(r)))
+    slip_mean = lambda g, r: float(np.mean(np.abs(g - r))) / float(np.max(np.abs(r)))
+    slip_den = lambda g, r: float(np.max(np.abs(g - r))) / float(np.max(np.abs(g)))
+    assert slip_abs(flip, ref) != O.scaled_max_err(flip, ref)
+    assert slip_mean(flip, ref) != O.scaled_max_err(flip, ref)
+    assert slip_den(np.array([2.0, 0.0]), np.array([1.0, 0.0])) != O.scaled_max_err(np.array([2.0, 0.0]), np.array([1.0, 0.0]))
+
+
+def test_max_row_rel_err_hand_cases():
+    ref = np.array([[3.0, 4.0], [0.0, 0.5], [300.0, 400.0]])            # row norms 5, 0.5, 500
+    assert O.max_row_rel_err(ref, ref) == 0.0
+    # the same absolute error (0.3, 0.4) -> norm 0.5 on each row in turn: 0.1, 1.0, 0.001 of the row
+    d = np.array([0.3, 0.4])
+    for r, want in ((0, 0.1), (1, 1.0), (2, 0.001)):
+        got = ref.copy(); got[r] += d
+        assert abs(O.max_row_rel_err(got, ref) - want) < 1e-15, r
+    # a small row off by a factor of two next to a large exact one: the coarse measure says 6e-4, this says 1
+    got = ref.copy(); got[1] *= 2.0
+    assert O.scaled_max_err(got, ref) == 0.5 / 400.0 and O.max_row_rel_err(got, ref) == 1.0
+    # a single entry that cancels to nearly zero does not dominate its row: error 0.05 on a row of norm 5
+    got = ref.copy(); got[0, 0] += 0.05
+    assert abs(O.max_row_rel_err(got, ref) - 0.01) < 1e-15
+    # scale from ref (not symmetric); a zero row has scale 1; 3-d input uses the last axis; empty -> 0
+    assert O.max_row_rel_err(np.array([[6.0, 8.0]]), np.array([[3.0, 4.0]])) == 1.0
+    assert O.max_row_rel_err(np.array([[3.0, 4.0]]), np.array([[6.0, 8.0]])) == 0.5
+    assert O.max_row_rel_err(np.array([[0.3, 0.4]]), np.zeros((1, 2))) == 0.5
+    assert O.max_row_rel_err(ref[None] * 1.0 + 0.0, ref[None]) == 0.0
+    assert O.max_row_rel_err(np.zeros((0, 4)), np.zeros((0, 4))) == 0.0
