@@ -50,6 +50,7 @@ extern "C" {
 #define STEM_ERR_TIMEOUT (-7)  /* device: a bounded pipeline wait expired          */
 #define STEM_ERR_ID_RANGE (-8) /* device: a token id was outside [0,V) (clamped)  */
 #define STEM_ERR_STATIC_LIMIT (-9) /* size beyond the fixed scratch of an allocation-free call */
+#define STEM_ERR_COUNT_RANGE (-10) /* device: a row count (device scalar) exceeded the buffers' capacity (clamped) */
 
 #define STEM_DTYPE_FP32 0
 #define STEM_DTYPE_BF16 1
@@ -88,7 +89,7 @@ int stem_workspace_bytes(const stem_shape_t* shape, size_t* bytes /*host, out*/)
 int stem_init_workspace(void* ws, size_t ws_bytes, void* stream);
 
 /* Synchronises `stream`, then copies the status word to *status_out (host):
- * STEM_OK, STEM_ERR_TIMEOUT or STEM_ERR_ID_RANGE.  The word is sticky: the first
+ * STEM_OK, STEM_ERR_TIMEOUT, STEM_ERR_ID_RANGE or STEM_ERR_COUNT_RANGE.  The word is sticky: the first
  * error stays until stem_init_workspace(). */
 int stem_query_status(const void* ws, void* stream, int32_t* status_out /*host*/);
 
@@ -153,6 +154,8 @@ int stem_ffn_forward(const stem_shape_t* shape, const void* x, const int32_t* id
  *   dW_down = dy^T H;  dW_gate = dG^T x;  dx = dG W_gate
  *   dE_rows[r] = sum of dU[t] over the positions t with ids[t] == unique_ids[r]
  *                (fixed summation order: the result is bitwise reproducible)
+ * When both weight gradients are asked for, the two token-contracted products run as one launch
+ * whose tiles share the SMs.
  * G_save, H_save: what stem_ffn_forward saved (required).  perm, seg_offsets, n_unique,
  * unique_ids: from stem_dedup_ids on the same ids.  dE_rows [min(T,V), d_ff]
  * (grad_dtype): rows >= n_u are left untouched; ids absent from the call have no row
@@ -197,7 +200,8 @@ int stem_dagger_backward(const stem_shape_t* shape, const void* dy, const void* 
  * checked, else STEM_ERR_NOT_PINNED) or in device memory (a compact on-device gather).
  * ids: device, normally unique_ids; n_ids: device scalar, so no host round trip is
  * needed between dedup and prefetch.  dev_cache: device [min(T,V), d_ff].  Run it on a
- * side stream to overlap the previous layer's GEMMs.
+ * side stream to overlap the previous layer's GEMMs.  A count outside [0, min(T,V)] is clamped
+ * to the cache's capacity and recorded in the status word as STEM_ERR_COUNT_RANGE (ws not NULL).
  */
 int stem_prefetch_rows(const stem_shape_t* shape, const int32_t* ids, const int32_t* n_ids,
                        const void* table, void* dev_cache, void* ws, void* stream);
@@ -250,7 +254,8 @@ int stem_lfu_refresh(const stem_shape_t* shape, int32_t K, const int32_t* freq, 
  *   *host_n = *n_rows.
  * host_rows [min(T,V), d_ff] (grad_dtype), host_ids [min(T,V)], host_n [1]: page-locked
  * host memory (checked).  The device writes them directly; they are complete once
- * `stream` has been synchronised.
+ * `stream` has been synchronised.  A count outside [0, min(T,V)] is clamped to that range (the
+ * host buffers hold no more); *host_n receives the clamped value.
  */
 int stem_writeback_rows(const stem_shape_t* shape, const void* dE_rows, const int32_t* unique_ids,
                         const int32_t* n_rows, void* host_rows, int32_t* host_ids,
@@ -354,10 +359,23 @@ int stem_ffn_step_host(const stem_shape_t* shape, const void* host_x, const int3
 int stem_ffn_step_host_flush(void* stream);
 
 /*
+ * Self-test of the device-side bounded wait (no counterpart in the paper).  Every wait inside
+ * the contraction kernels (on a TMA copy, on the tensor cores, on the epilogue) gives up after
+ * a cycle limit, records STEM_ERR_TIMEOUT in the status word and lets the kernel unwind instead
+ * of hanging the GPU.  This call runs that wait alone: one thread of one small CTA waits on a
+ * barrier for at most limit_cycles SM clocks (1 .. 2e9).  arrive == 0: nothing ever completes the
+ * barrier, the wait runs out, stem_query_status(ws) then returns STEM_ERR_TIMEOUT (detail 100)
+ * and stem_init_workspace re-arms the word.  arrive != 0: the barrier is completed first, the
+ * wait succeeds and the status stays as it was.  No copy or MMA is in flight either way; the
+ * kernel always returns.  ws: an initialised workspace (status word only).
+ */
+int stem_selftest_wait(void* ws, long long limit_cycles, int arrive, void* stream);
+
+/*
  * Instrumentation (no counterpart in the paper).  stem_launch_count: kernels this library
  * has launched in this process.  stem_profile_enable(1) clears earlier records and starts
  * recording one CUDA-event pair per step of the path (dedup, gate_gemm, down_gemm,
- * dh_gemm, dw_down_gemm, seg_reduce, dw_gate_gemm, dx_gemm, prefetch_rows,
+ * dh_gemm, seg_reduce, dw_pair_gemm (or dw_down_gemm, dw_gate_gemm), dx_gemm, prefetch_rows,
  * writeback_rows, h2d_inputs, d2h_outputs) on the stream of each call; (0) stops.
  * stem_profile_get waits for record i to finish and returns its name (static storage) and
  * its duration in milliseconds.

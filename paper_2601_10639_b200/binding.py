@@ -21,6 +21,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_ARCH = -1, -2, -3
 ERR_WORKSPACE_TOO_SMALL, ERR_NOT_PINNED, ERR_CUDA, ERR_TIMEOUT, ERR_ID_RANGE = -4, -5, -6, -7, -8
 ERR_STATIC_LIMIT = -9
+ERR_COUNT_RANGE = -10
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 FLAG_SIMT = 1
 FLAG_SINGLE_CTA = 2
@@ -33,6 +34,7 @@ EXPORTS = (
     "stem_ffn_step_host", "stem_ffn_step_host_flush", "stem_launch_count", "stem_profile_enable", "stem_profile_count", "stem_profile_get",
     "stem_dedup_ids_static", "stem_dedup_static_max_tokens",
     "stem_shard_route_workspace_bytes", "stem_shard_route", "stem_reduce_rows", "stem_gather_rows",
+    "stem_selftest_wait",
 )
 
 
@@ -89,6 +91,7 @@ def lib() -> ctypes.CDLL:
             "stem_shard_route": [i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp],
             "stem_reduce_rows": [shp, vp, vp, vp, vp, vp, vp, sz, vp],
             "stem_gather_rows": [shp, vp, vp, vp, vp, vp, vp],
+            "stem_selftest_wait": [vp, ctypes.c_longlong, ctypes.c_int, vp],
             "stem_profile_enable": [ctypes.c_int],
             "stem_profile_count": [],
             "stem_profile_get": [ctypes.c_int, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float)],
@@ -268,6 +271,10 @@ def stem_gather_rows(shape, ids, n_ids, table, out, ws=None, stream=None) -> Non
 def stem_reduce_rows(shape, rows_in, perm, seg_offsets, n_unique, rows_out, ws, stream=None) -> None:
     _check(lib().stem_reduce_rows(ctypes.byref(shape), _p(rows_in), _p(perm), _p(seg_offsets), _p(n_unique),
                                   _p(rows_out), _p(ws), ws.numel(), _stream(stream)), "stem_reduce_rows")
+
+
+def stem_selftest_wait(ws, limit_cycles: int, arrive: bool, stream=None) -> None:
+    _check(lib().stem_selftest_wait(_p(ws), int(limit_cycles), 1 if arrive else 0, _stream(stream)), "stem_selftest_wait")
 
 
 def stem_launch_count() -> int:

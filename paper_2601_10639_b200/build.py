@@ -10,7 +10,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libstem.so")
-SOURCES = ["api.cu", "gemm_sm100.cu", "simt_gemm.cu", "dedup.cu", "segreduce.cu", "rows.cu", "lfu.cu", "shard.cu"]
+SOURCES = ["api.cu", "gemm_sm100.cu", "simt_gemm.cu", "dedup.cu", "segreduce.cu", "rows.cu", "lfu.cu", "shard.cu", "selftest.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC"]
 

@@ -182,6 +182,7 @@ const char* stem_status_string(int code) {
     case STEM_ERR_CUDA: return g_cuda_msg[0] ? g_cuda_msg : "CUDA error";
     case STEM_ERR_TIMEOUT: return "device: a bounded pipeline wait expired";
     case STEM_ERR_ID_RANGE: return "device: token id outside [0,V) (clamped)";
+    case STEM_ERR_COUNT_RANGE: return "device: a row count exceeded the capacity of the row buffers (clamped)";
     case STEM_ERR_STATIC_LIMIT: return "size exceeds the fixed scratch of the allocation-free entry point (T > 65536)";
     default: return "unknown status";
   }
@@ -295,27 +296,37 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
     e = gemm(shape, T, F, d, dy, false, W_down, true, kEpiDH, dh, st);
   }
   if (e != cudaSuccess) return cuda_fail(e);
-  if (dW_down) {  // dW_down[i,j] = sum_t dy[t,i] H[t,j]
-    EpiParams p; p.out = dW_down; p.out_fp32 = grad_fp32; p.status = status_of(ws);
-    p.accumulate = (shape->flags & STEM_FLAG_ACCUM_GRADS) != 0;
-    p.sk_scratch = base + w.sk_off; p.sk_bytes = w.sk_bytes;
-    ProfScope prof("dw_down_gemm", st);
-    e = gemm(shape, d, F, T, dy, true, H_save, true, kEpiStore, p, st);
-    if (e != cudaSuccess) return cuda_fail(e);
-  }
+  // Table gradient first: the tail of dU is still in L2 behind the dH kernel.
   if (dE_rows) {
     ProfScope prof("seg_reduce", st);
     e = launch_segreduce(T, F, shape->dtype, shape->grad_dtype, dU, perm, seg_offsets, n_unique, dE_rows,
                          base + w.part_off, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
-  if (dW_gate) {  // dW_gate[j,k] = sum_t dG[t,j] x[t,k]
-    EpiParams p; p.out = dW_gate; p.out_fp32 = grad_fp32; p.status = status_of(ws);
-    p.accumulate = (shape->flags & STEM_FLAG_ACCUM_GRADS) != 0;
-    p.sk_scratch = base + w.sk_off; p.sk_bytes = w.sk_bytes;
-    ProfScope prof("dw_gate_gemm", st);
-    e = gemm(shape, F, d, T, dG, true, x, true, kEpiStore, p, st);
+  EpiParams gp; gp.out_fp32 = grad_fp32; gp.status = status_of(ws);
+  gp.accumulate = (shape->flags & STEM_FLAG_ACCUM_GRADS) != 0;
+  gp.sk_scratch = base + w.sk_off; gp.sk_bytes = w.sk_bytes;
+  if (dW_down && dW_gate && use_tc(shape)) {
+    // dW_down[i,j] = sum_t dy[t,i] H[t,j] and dW_gate[j,k] = sum_t dG[t,j] x[t,k] in ONE launch: both
+    // contract over the tokens, and their output tiles together fill the SMs (at the 350M shape
+    // each has 44 tiles for 74 CTA pairs) with one split tail and one fix-up instead of two
+    ProfScope prof("dw_pair_gemm", st);
+    e = launch_tc_gemm_token_pair(T, d, F, dy, H_save, dW_down, F, d, dG, x, dW_gate, gp,
+                                  !(shape->flags & STEM_FLAG_SINGLE_CTA), st);
     if (e != cudaSuccess) return cuda_fail(e);
+  } else {
+    if (dW_down) {  // dW_down[i,j] = sum_t dy[t,i] H[t,j]
+      EpiParams p = gp; p.out = dW_down;
+      ProfScope prof("dw_down_gemm", st);
+      e = gemm(shape, d, F, T, dy, true, H_save, true, kEpiStore, p, st);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (dW_gate) {  // dW_gate[j,k] = sum_t dG[t,j] x[t,k]
+      EpiParams p = gp; p.out = dW_gate;
+      ProfScope prof("dw_gate_gemm", st);
+      e = gemm(shape, F, d, T, dG, true, x, true, kEpiStore, p, st);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
   }
   if (dx) {  // dx = dG W_gate (contraction over d_ff; W_gate is [F, d]: d contiguous)
     EpiParams p; p.out = dx; p.out_fp32 = shape->dtype == STEM_DTYPE_FP32; p.status = status_of(ws);
@@ -574,7 +585,8 @@ int stem_writeback_rows(const stem_shape_t* shape, const void* dE_rows, const in
   ProfScope prof("writeback_rows", static_cast<cudaStream_t>(stream));
   cudaError_t e = launch_writeback_rows(max_rows, row_bytes, dE_rows, unique_ids, n_rows, const_cast<void*>(hr),
                                         static_cast<int32_t*>(const_cast<void*>(hi)),
-                                        static_cast<int32_t*>(const_cast<void*>(hn)), static_cast<cudaStream_t>(stream));
+                                        static_cast<int32_t*>(const_cast<void*>(hn)), nullptr,
+                                        static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
 }
 
@@ -615,6 +627,13 @@ int stem_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int32_t a_mn,
   return e == cudaSuccess ? STEM_OK : cuda_fail(e);
 }
 
+int stem_selftest_wait(void* ws, long long limit_cycles, int arrive, void* stream) {
+  if (!ws || !aligned16(ws)) return STEM_ERR_INVALID_ARG;
+  if (limit_cycles < 1 || limit_cycles > 2000000000ll) return STEM_ERR_INVALID_ARG;
+  cudaError_t e = launch_selftest_wait(status_of(ws), limit_cycles, arrive, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? STEM_OK : cuda_fail(e);
+}
+
 long long stem_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int stem_profile_enable(int on) {
@@ -652,7 +671,7 @@ namespace {
 // TWO slots of input (x, dy, ids) and output (y, dx) buffers, so the copies of one call
 // overlap the kernels of its neighbours.
 struct Arena {
-  size_t ws, ws_bytes, x[2], dy[2], ids[2], y[2], dx[2], G, H, inverse, perm, seg, total;
+  size_t ws, ws_bytes, x[2], dy[2], ids[2], y[2], dx[2], n_u[2], G, H, inverse, perm, seg, total;
 };
 Arena arena_layout(const stem_shape_t* s) {
   Arena a{};
@@ -664,6 +683,7 @@ Arena arena_layout(const stem_shape_t* s) {
   for (int k = 0; k < 2; ++k) {
     a.x[k] = o; o += td;  a.dy[k] = o; o += td;  a.ids[k] = o; o += ti;
     a.y[k] = o; o += td;  a.dx[k] = o; o += td;
+    a.n_u[k] = o; o += 256;   // this call's row count, kept until its copy to the host has run
   }
   a.G = o; o += tf;  a.H = o; o += tf;
   a.inverse = o; o += ti;  a.perm = o; o += ti;  a.seg = o; o += align_up((R + 1) * 4, 256);
@@ -754,6 +774,10 @@ int stem_ffn_step_host(const stem_shape_t* shape, const void* host_x, const int3
   if (int rc = stem_ffn_backward(shape, base + a.dy[k], base + a.x[k], ids, W_gate, E, W_down, base + a.G, base + a.H,
                                  perm, seg, n_unique, base + a.dx[k], dW_gate, dW_down, dE_rows, unique_ids,
                                  base + a.ws, a.ws_bytes, stream)) return rc;
+  // The caller's n_unique scalar is rewritten by the next call's dedup long before this call's
+  // output copies run: the count that goes to the host is taken from a word of this slot (copied
+  // here, behind the last kernel, where the stream has an event boundary anyway).
+  if (host_n_unique) STEP_CUDA(cudaMemcpyAsync(base + a.n_u[k], n_unique, 4, cudaMemcpyDeviceToDevice, st));
   STEP_CUDA(cudaEventRecord(p.bwd_done[k], st));
   // outputs
   STEP_CUDA(cudaStreamWaitEvent(p.out, p.y_done[k], 0));
@@ -762,7 +786,7 @@ int stem_ffn_step_host(const stem_shape_t* shape, const void* host_x, const int3
     STEP_CUDA(cudaMemcpyAsync(host_y, base + a.y[k], td, cudaMemcpyDeviceToHost, p.out));
     STEP_CUDA(cudaStreamWaitEvent(p.out, p.bwd_done[k], 0));
     STEP_CUDA(cudaMemcpyAsync(host_dx, base + a.dx[k], td, cudaMemcpyDeviceToHost, p.out));
-    if (host_n_unique) STEP_CUDA(cudaMemcpyAsync(host_n_unique, n_unique, 4, cudaMemcpyDeviceToHost, p.out));
+    if (host_n_unique) STEP_CUDA(cudaMemcpyAsync(host_n_unique, base + a.n_u[k], 4, cudaMemcpyDeviceToHost, p.out));
   }
   STEP_CUDA(cudaEventRecord(p.out_done[k], p.out));
   p.used[k] = true;

@@ -70,25 +70,41 @@ __device__ __forceinline__ float fast_sigmoid(float g) {
 // ---- 32-column row segments: global <-> registers -------------------------------------
 // WIDE: the row pitch and base are multiples of 32 bytes, so 256-bit accesses are legal and
 // a 16-column group is wholly inside or outside the matrix.  Otherwise 128-bit accesses.
+// NC: the memory is read-only for the whole kernel, so the non-coherent path may serve it.  The
+// add epilogue can run in place (its addend is the buffer it overwrites): it reads with plain
+// loads.
+template <bool NC>
 __device__ __forceinline__ void ldg256(const void* p, uint32_t* r) {
-  asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "l"(p));
+  if (NC) {
+    asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "l"(p));
+  } else {
+    asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "l"(p) : "memory");
+  }
 }
+template <bool NC>
 __device__ __forceinline__ void ldg128(const void* p, uint32_t* r) {
-  const uint4 q = __ldg(static_cast<const uint4*>(p));
+  uint4 q;
+  if (NC) {
+    q = __ldg(static_cast<const uint4*>(p));
+  } else {
+    asm volatile("ld.global.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w) : "l"(p) : "memory");
+  }
   r[0] = q.x; r[1] = q.y; r[2] = q.z; r[3] = q.w;
 }
 
 // 32 bf16 (16 registers) starting at column n of a row; p points at column n.
-template <bool WIDE>
+template <bool WIDE, bool NC = true>
 __device__ __forceinline__ void load_bf16x32(const __nv_bfloat16* p, int n, int N, uint32_t (&r)[16]) {
   if (WIDE) {
 #pragma unroll
-    for (int h = 0; h < 2; ++h) if (n + 16 * h < N) ldg256(p + 16 * h, r + 8 * h);
+    for (int h = 0; h < 2; ++h) if (n + 16 * h < N) ldg256<NC>(p + 16 * h, r + 8 * h);
   } else {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) if (n + 8 * q < N) ldg128(p + 8 * q, r + 4 * q);
+    for (int q = 0; q < 4; ++q) if (n + 8 * q < N) ldg128<NC>(p + 8 * q, r + 4 * q);
   }
 }
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -203,7 +219,9 @@ template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE, int CTA
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
-               int M, int N, int K, int group_m, int dp_tiles, int split, EpiParams ep) {
+               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
+               const __grid_constant__ CUtensorMap tmC2,
+               int M, int N, int K, int M2, int N2, int group_m, int dp_tiles, int split, EpiParams ep) {
   using L = Smem<BN, STAGES, CTAS>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -223,7 +241,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t rank = CTAS == 2 ? ptx::cluster_ctarank() : 0u;
   const int unit0 = blockIdx.x / CTAS, unit_stride = gridDim.x / CTAS;
   const int tiles_m = (M + BM * CTAS - 1) / (BM * CTAS), tiles_n = (N + BN - 1) / BN;
-  const int num_tiles = tiles_m * tiles_n;
+  // A second product with the same contraction length may ride in the same launch (plain stores
+  // only): its tiles are numbered after the first product's and share one work list, so the two
+  // fill the machine together where each alone would leave SMs idle.
+  const int tiles_m2 = KIND == kEpiStore && M2 > 0 ? (M2 + BM * CTAS - 1) / (BM * CTAS) : 0;
+  const int tiles_n2 = KIND == kEpiStore && M2 > 0 ? (N2 + BN - 1) / BN : 0;
+  const int num_tiles1 = tiles_m * tiles_n;
+  const int num_tiles = num_tiles1 + tiles_m2 * tiles_n2;
   const int k_blocks = (K + BK - 1) / BK;
   constexpr uint32_t kTmemCols = 2 * BN;
   const WorkList work{unit0, unit_stride, dp_tiles, num_tiles, k_blocks, split};
@@ -238,6 +262,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ptx::prefetch_tensormap(&tmB);
     ptx::prefetch_tensormap(&tmC0);
     if (KIND == kEpiGate || KIND == kEpiDH) ptx::prefetch_tensormap(&tmC1);
+    if (KIND == kEpiStore && M2 > 0) {
+      ptx::prefetch_tensormap(&tmA2);
+      ptx::prefetch_tensormap(&tmB2);
+      ptx::prefetch_tensormap(&tmC2);
+    }
   }
   if (warp == 1) {
     if (CTAS == 2) {
@@ -266,7 +295,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       Work w;
       for (int i = 0; ok && work.get(i, w); ++i) {
-        const TileCoord tc = tile_coord(w.tile, tiles_m, tiles_n, group_m);
+        const bool second = KIND == kEpiStore && w.tile >= num_tiles1;
+        const TileCoord tc = second ? tile_coord(w.tile - num_tiles1, tiles_m2, tiles_n2, group_m)
+                                    : tile_coord(w.tile, tiles_m, tiles_n, group_m);
+        const CUtensorMap* mapA = second ? &tmA2 : &tmA;
+        const CUtensorMap* mapB = second ? &tmB2 : &tmB;
         // this CTA's rows of A and its share of the columns of B
         const int m0 = (tc.m_blk * CTAS + rank) * BM, n0 = tc.n_blk * BN + rank * (BN / CTAS);
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
@@ -285,15 +318,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const int k0 = kb * BK;
           if (A_MN) {
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j) load(a_dst + j * kAtomBytes, &tmA, m0 + 64 * j, k0);
+            for (int j = 0; j < BM / 64; ++j) load(a_dst + j * kAtomBytes, mapA, m0 + 64 * j, k0);
           } else {
-            load(a_dst, &tmA, k0, m0);
+            load(a_dst, mapA, k0, m0);
           }
           if (B_MN) {
 #pragma unroll
-            for (int j = 0; j < BN / CTAS / 64; ++j) load(b_dst + j * kAtomBytes, &tmB, n0 + 64 * j, k0);
+            for (int j = 0; j < BN / CTAS / 64; ++j) load(b_dst + j * kAtomBytes, mapB, n0 + 64 * j, k0);
           } else {
-            load(b_dst, &tmB, k0, n0);
+            load(b_dst, mapB, k0, n0);
           }
           ++issued;
           if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -357,15 +390,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr int kChunks = BN / 2 / 32;    // 32-column chunks per thread per tile
     const uint32_t out_buf = base + L::kOutOffset + (warp - 2) * L::kOutBytesPerWarp;
     const bool second_out = KIND == kEpiDH || (KIND == kEpiGate && ep.G != nullptr);
+    constexpr bool kReadOnlyE = KIND != kEpiAdd;   // the add epilogue may overwrite its addend
     int acc = 0; uint32_t aph = 0;
     bool ok = true;
     Work w;
     for (int i = 0; ok && work.get(i, w); ++i) {
-      const TileCoord tc = tile_coord(w.tile, tiles_m, tiles_n, group_m);
+      const bool second = KIND == kEpiStore && w.tile >= num_tiles1;
+      const TileCoord tc = second ? tile_coord(w.tile - num_tiles1, tiles_m2, tiles_n2, group_m)
+                                  : tile_coord(w.tile, tiles_m, tiles_n, group_m);
+      const CUtensorMap* mapC = second ? &tmC2 : &tmC0;
+      const int M_ = second ? M2 : M, N_ = second ? N2 : N;    // extents of the product this tile belongs to
       const int m_warp = (tc.m_blk * CTAS + rank) * BM + q * 32;  // first row of this warp's 32-row block
       const int m = m_warp + lane;
       const int n0 = tc.n_blk * BN + half * (BN / 2);
-      const bool row_ok = m < M;
+      const bool row_ok = m < M_;
       const size_t row_off = static_cast<size_t>(m) * N;
       const __nv_bfloat16* e_row = nullptr;
       const __nv_bfloat16* g_row = nullptr;
@@ -381,7 +419,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // operands of the first chunk are requested before waiting for the accumulator
       uint32_t e_next[16], g_next[16];
       if (KIND != kEpiStore && row_ok) {
-        load_bf16x32<WIDE>(e_row + n0, n0, N, e_next);
+        load_bf16x32<WIDE, kReadOnlyE>(e_row + n0, n0, N, e_next);
         if (KIND == kEpiDH) load_bf16x32<WIDE>(g_row + n0, n0, N, g_next);
       }
       bool mine = ptx::mbar_wait_bounded(tfull_bar(acc), aph, abort_flag, kWaitLimitCycles);
@@ -399,7 +437,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int i = 0; i < 16; ++i) { e_cur[i] = e_next[i]; g_cur[i] = g_next[i]; }
         const int n = n0 + c * 32;
         if (KIND != kEpiStore && row_ok && c + 1 < kChunks) {
-          load_bf16x32<WIDE>(e_row + n + 32, n + 32, N, e_next);
+          load_bf16x32<WIDE, kReadOnlyE>(e_row + n + 32, n + 32, N, e_next);
           if (KIND == kEpiDH) load_bf16x32<WIDE>(g_row + n + 32, n + 32, N, g_next);
         }
         uint32_t v[32];
@@ -430,9 +468,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           epilogue_row32<KIND>(ep, out_buf, lane, v, e_cur, g_cur);
           ptx::fence_proxy_async();
           __syncwarp();
-          if (lane == 0 && m_warp < M && n < N) {
-            if (KIND == kEpiStore && ep.accumulate) ptx::tma_reduce_add_2d(&tmC0, out_buf, n, m_warp);
-            else ptx::tma_store_2d(&tmC0, out_buf, n, m_warp);
+          if (lane == 0 && m_warp < M_ && n < N_) {
+            if (KIND == kEpiStore && ep.accumulate) ptx::tma_reduce_add_2d(mapC, out_buf, n, m_warp);
+            else ptx::tma_store_2d(mapC, out_buf, n, m_warp);
             if (second_out) ptx::tma_store_2d(&tmC1, out_buf + 2048, n, m_warp);
             ptx::bulk_commit_group();
           }
@@ -481,12 +519,18 @@ constexpr int kFixRows = 8;    // rows of a tile per fix-up CTA
 template <int BN, int CTAS>
 __global__ void __launch_bounds__(256)
 tail_fixup_kernel(int M, int N, int dp_tiles, int tail, int split, int tiles_m, int tiles_n, int group_m,
-                  const float* __restrict__ partial, void* __restrict__ out, int out_fp32, int accumulate) {
+                  const float* __restrict__ partial, void* __restrict__ out, int out_fp32, int accumulate,
+                  int M2, int N2, int tiles_m2, int tiles_n2, void* __restrict__ out2) {
   constexpr int TM = BM * CTAS;
   ptx::grid_dependency_wait();
   ptx::grid_launch_dependents();
   const int j = blockIdx.x;
-  const TileCoord tc = tile_coord(dp_tiles + j, tiles_m, tiles_n, group_m);
+  // tiles of a second product riding in the same launch are numbered after the first product's
+  const int num_tiles1 = tiles_m * tiles_n;
+  const bool second = dp_tiles + j >= num_tiles1;
+  const TileCoord tc = second ? tile_coord(dp_tiles + j - num_tiles1, tiles_m2, tiles_n2, group_m)
+                              : tile_coord(dp_tiles + j, tiles_m, tiles_n, group_m);
+  if (second) { M = M2; N = N2; out = out2; }
   const int r0 = blockIdx.y * kFixRows;
   for (int e = threadIdx.x; e < kFixRows * (BN / 4); e += 256) {
     const int r = r0 + e / (BN / 4), c = (e % (BN / 4)) * 4;
@@ -571,10 +615,14 @@ bool encode_out_map(CUtensorMap* map, const void* ptr, int rows, int cols, bool 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A second product C2 = A2 B2^T with the same contraction length and operand layouts, carried by
+// the same launch (plain stores only); M == 0 means none.
+struct SecondMaps { CUtensorMap A, B, C; int M = 0, N = 0; void* out = nullptr; };
+
 template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE, int CTAS>
 cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC0,
                         const CUtensorMap& tmC1, int M, int N, int K, const EpiParams& ep, int sk_tail,
-                        int sk_split, cudaStream_t stream) {
+                        int sk_split, const SecondMaps& sec, cudaStream_t stream) {
   using L = Smem<BN, STAGES, CTAS>;
   static_assert(L::kTotal <= 232448, "exceeds the shared memory a CTA can have");
   auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES, WIDE, CTAS>;
@@ -585,7 +633,8 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     return ce;
   // persistent: one CTA (or one pair) per SM (pair of SMs), each walking its work list
   const int tiles_m = (M + BM * CTAS - 1) / (BM * CTAS), tiles_n = (N + BN - 1) / BN;
-  const int units = tiles_m * tiles_n;
+  const int tiles_m2 = sec.M > 0 ? (sec.M + BM * CTAS - 1) / (BM * CTAS) : 0, tiles_n2 = sec.M > 0 ? (sec.N + BN - 1) / BN : 0;
+  const int units = tiles_m * tiles_n + tiles_m2 * tiles_n2;
   const int slots = device_sm_count() / CTAS;
   const int P = sk_tail > 0 ? slots : (units < slots ? units : slots);
   const int dp_tiles = sk_tail > 0 ? units - sk_tail : units;
@@ -603,7 +652,8 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC0, tmC1, M, N, K, 8, dp_tiles, sk_split, ep);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC0, tmC1, sec.M > 0 ? sec.A : tmA, sec.M > 0 ? sec.B : tmB,
+                                     sec.M > 0 ? sec.C : tmC0, M, N, K, sec.M, sec.N, 8, dp_tiles, sk_split, ep);
   count_launches(1);
   if (e == cudaSuccess && sk_tail > 0) {
     cudaLaunchConfig_t fcfg = {};
@@ -614,15 +664,17 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
     fcfg.numAttrs = 1;
     e = cudaLaunchKernelEx(&fcfg, tail_fixup_kernel<BN, CTAS>, M, N, dp_tiles, sk_tail, sk_split, tiles_m, tiles_n, 8,
                            static_cast<const float*>(ep.sk_scratch), ep.out, static_cast<int>(ep.out_fp32),
-                           static_cast<int>(ep.accumulate));
+                           static_cast<int>(ep.accumulate), sec.M, sec.N, tiles_m2, tiles_n2, sec.out);
     count_launches(1);
   }
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
+struct SecondProduct { int M = 0, N = 0; const void* A = nullptr; const void* B = nullptr; void* out = nullptr; };
+
 template <bool A_MN, bool B_MN, int KIND, int CTAS>
 cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const EpiParams& ep,
-                      cudaStream_t stream) {
+                      const SecondProduct& second, cudaStream_t stream) {
   // 192 KB of operand ring either way: 4 stages of 48 KB, or 6 stages of 32 KB per CTA of a pair
   constexpr int BN = 256, STAGES = CTAS == 2 ? 6 : 4;
   CUtensorMap tmA, tmB;
@@ -630,16 +682,24 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
   const bool okB = B_MN ? encode_map(&tmB, B, K, N, BK) : encode_map(&tmB, B, N, K, BN / CTAS);
   if (!okA || !okB) return cudaErrorNotSupported;
   CUtensorMap tmC0, tmC1;
+  SecondMaps sec;
   bool okC;
   int sk_tail = 0, sk_split = 1;  // tiles of the ragged last round, pieces per tile along k
   if (KIND == kEpiStore) {
     okC = encode_out_map(&tmC0, ep.out, M, N, ep.out_fp32 != 0);
     tmC1 = tmC0;
+    if (second.M > 0) {
+      sec.M = second.M; sec.N = second.N; sec.out = second.out;
+      okC = okC && (A_MN ? encode_map(&sec.A, second.A, K, second.M, BK) : encode_map(&sec.A, second.A, second.M, K, BM));
+      okC = okC && (B_MN ? encode_map(&sec.B, second.B, K, second.N, BK) : encode_map(&sec.B, second.B, second.N, K, BN / CTAS));
+      okC = okC && encode_out_map(&sec.C, second.out, second.M, second.N, ep.out_fp32 != 0);
+    }
     // The last round costs ceil(tail * split / slots) / split tile times instead of one.
     // Worth it when that saves clearly more than the partial tiles and the fix-up launch
     // cost (10-25 us together); a tile time is ~ 2 TM BN K flops at ~11 TFLOP/s per SM.
     constexpr int TM = BM * CTAS;
-    const int units = ((M + TM - 1) / TM) * ((N + BN - 1) / BN);
+    const int units = ((M + TM - 1) / TM) * ((N + BN - 1) / BN) +
+                      (second.M > 0 ? ((second.M + TM - 1) / TM) * ((second.N + BN - 1) / BN) : 0);
     const int slots = device_sm_count() / CTAS;
     const int k_blocks = (K + BK - 1) / BK;
     const int tail = units % slots;
@@ -666,18 +726,31 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
   if (!okC) return cudaErrorNotSupported;
   auto a32 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; };
   const bool wide = (N % 16 == 0) && a32(ep.E) && a32(ep.Gin);
-  if (wide) return launch_inst<A_MN, B_MN, KIND, BN, STAGES, true, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, sk_tail, sk_split, stream);
-  return launch_inst<A_MN, B_MN, KIND, BN, STAGES, false, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, sk_tail, sk_split, stream);
+  if (wide) return launch_inst<A_MN, B_MN, KIND, BN, STAGES, true, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, sk_tail, sk_split, sec, stream);
+  return launch_inst<A_MN, B_MN, KIND, BN, STAGES, false, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, sk_tail, sk_split, sec, stream);
 }
 
 template <bool A_MN, bool B_MN, int KIND>
 cudaError_t launch_ctas(const void* A, const void* B, int M, int N, int K, const EpiParams& ep, bool pair,
                         cudaStream_t stream) {
-  if (pair) return launch_bn<A_MN, B_MN, KIND, 2>(A, B, M, N, K, ep, stream);
-  return launch_bn<A_MN, B_MN, KIND, 1>(A, B, M, N, K, ep, stream);
+  if (pair) return launch_bn<A_MN, B_MN, KIND, 2>(A, B, M, N, K, ep, SecondProduct{}, stream);
+  return launch_bn<A_MN, B_MN, KIND, 1>(A, B, M, N, K, ep, SecondProduct{}, stream);
 }
 
 }  // namespace
+
+cudaError_t launch_tc_gemm_token_pair(int K, int M1, int N1, const void* A1, const void* B1, void* out1, int M2,
+                                      int N2, const void* A2, const void* B2, void* out2, const EpiParams& ep,
+                                      bool pair, cudaStream_t stream) {
+  if (K <= 0 || M1 <= 0 || N1 <= 0 || M2 <= 0 || N2 <= 0) return cudaErrorNotSupported;
+  if ((M1 % 8) || (N1 % 8) || (M2 % 8) || (N2 % 8)) return cudaErrorNotSupported;
+  EpiParams p = ep;
+  p.out = out1;
+  SecondProduct second;
+  second.M = M2; second.N = N2; second.A = A2; second.B = B2; second.out = out2;
+  if (pair) return launch_bn<true, true, kEpiStore, 2>(A1, B1, M1, N1, K, p, second, stream);
+  return launch_bn<true, true, kEpiStore, 1>(A1, B1, M1, N1, K, p, second, stream);
+}
 
 size_t tc_gemm_scratch_bytes() {
   // room for 296 partial 256 x 256 fp32 tiles: up to four pieces for each of the at most 73

@@ -89,10 +89,12 @@ lfu_lists_kernel(int K, const int32_t* __restrict__ ranking, const uint8_t* __re
 // Entering id i takes free slot i; its row is copied from the table (host memory: 16-byte
 // loads across the host link, eight in flight per thread).
 __global__ void __launch_bounds__(kCopyThreads)
-lfu_install_kernel(int vec_per_row, const int32_t* __restrict__ counts, const int32_t* __restrict__ free_slots,
+lfu_install_kernel(int K, int vec_per_row, const int32_t* __restrict__ counts, const int32_t* __restrict__ free_slots,
                    const int32_t* __restrict__ entering, const uint4* __restrict__ table,
                    int32_t* hot_slot, int32_t* hot_ids, uint4* __restrict__ hot_rows, int32_t* n_installed) {
-  const int n = counts[1];   // never more than counts[0]: the cache has K slots and the new set at most K ids
+  // never more than counts[0] (the cache has K slots and the new set at most K ids); bounded all
+  // the same, so that no count can carry a copy past the K rows of the cache
+  const int n = min(min(counts[1], counts[0]), K);
   if (blockIdx.x == 0 && threadIdx.x == 0 && n_installed != nullptr) *n_installed = n;
   for (int i = blockIdx.x; i < n; i += gridDim.x) {
     const int slot = free_slots[i], id = entering[i];
@@ -161,7 +163,7 @@ cudaError_t launch_lfu_refresh(int V, int K, size_t row_bytes, const int32_t* fr
   lfu_mark_kernel<<<kblocks, kThreads, 0, stream>>>(K, ranking, freq, in_new);
   lfu_lists_kernel<<<kblocks, kThreads, 0, stream>>>(K, ranking, in_new, hot_slot, hot_ids, free_slots, entering, counts);
   lfu_install_kernel<<<kCopyCtas, kCopyThreads, 0, stream>>>(
-      static_cast<int>(row_bytes / 16), counts, free_slots, entering, static_cast<const uint4*>(table), hot_slot,
+      K, static_cast<int>(row_bytes / 16), counts, free_slots, entering, static_cast<const uint4*>(table), hot_slot,
       hot_ids, static_cast<uint4*>(hot_rows), n_installed);
   count_launches(4);
   return cudaGetLastError();

@@ -19,11 +19,16 @@ constexpr int kHostLinkCtas = 32;
 constexpr int kHostLinkThreads = 128;
 
 __global__ void __launch_bounds__(kThreads)
-gather_rows_kernel(int V, int vec_per_row, const int32_t* __restrict__ ids,
+gather_rows_kernel(int max_rows, int V, int vec_per_row, const int32_t* __restrict__ ids,
                    const int32_t* __restrict__ n_ids, const uint4* __restrict__ table,
                    const uint4* __restrict__ hot_rows, const int32_t* __restrict__ hot_slot,
                    uint4* __restrict__ dst, int32_t* status, int32_t* stats) {
-  const int n = *n_ids;
+  // the count is a device scalar the host never saw: never trust it beyond the buffers' capacity
+  int n = *n_ids;
+  if (n > max_rows || n < 0) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) report_error(status, STEM_ERR_COUNT_RANGE, n);
+    n = n < 0 ? 0 : max_rows;
+  }
   // a CTA handles `rows_per_cta` rows per step so short rows still fill the block
   const int lanes_per_row = min(vec_per_row, static_cast<int>(blockDim.x));
   const int rows_per_cta = static_cast<int>(blockDim.x) / lanes_per_row;
@@ -59,12 +64,77 @@ gather_rows_kernel(int V, int vec_per_row, const int32_t* __restrict__ ids,
   }
 }
 
+// Device-resident table (and hot set): the whole copy is one flat list of 16-byte vectors,
+// vector i belonging to row i / vec_per_row, dealt to the threads in batches of kFlatBatch with
+// the next batch's loads issued before the current batch is stored.  No thread ever waits on a
+// row's id before it can ask for the row: every vector looks its id up itself (one cached 4-byte
+// load shared by the whole row), so the id -> row address -> data chains of 2 * kFlatBatch
+// vectors per thread overlap.
+constexpr int kFlatBatch = 4;
+
+__device__ __forceinline__ const uint4* flat_src(size_t i, int vec_per_row, int V, const int32_t* __restrict__ ids,
+                                                 const uint4* __restrict__ table, const uint4* __restrict__ hot_rows,
+                                                 const int32_t* __restrict__ hot_slot, int32_t* status, int32_t* stats) {
+  // 32-bit division whenever the index allows (it nearly always does): far cheaper than 64-bit
+  const int r = (i >> 32) == 0 ? static_cast<int>(static_cast<uint32_t>(i) / static_cast<uint32_t>(vec_per_row))
+                               : static_cast<int>(i / vec_per_row);
+  const int c = static_cast<int>(i - static_cast<size_t>(r) * vec_per_row);
+  int id = __ldg(ids + r);
+  if (id < 0 || id >= V) {
+    if (c == 0) report_error(status, STEM_ERR_ID_RANGE, r);
+    id = id < 0 ? 0 : V - 1;
+  }
+  const int slot = hot_slot != nullptr ? __ldg(hot_slot + id) : -1;
+  if (stats != nullptr && c == 0) atomicAdd(stats + (slot >= 0 ? 0 : 1), 1);
+  return (slot >= 0 ? hot_rows + static_cast<size_t>(slot) * vec_per_row : table + static_cast<size_t>(id) * vec_per_row) + c;
+}
+
+__global__ void __launch_bounds__(kThreads)
+gather_rows_flat_kernel(int max_rows, int V, int vec_per_row, const int32_t* __restrict__ ids,
+                        const int32_t* __restrict__ n_ids, const uint4* __restrict__ table,
+                        const uint4* __restrict__ hot_rows, const int32_t* __restrict__ hot_slot,
+                        uint4* __restrict__ dst, int32_t* status, int32_t* stats) {
+  int n = *n_ids;
+  if (n > max_rows || n < 0) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) report_error(status, STEM_ERR_COUNT_RANGE, n);
+    n = n < 0 ? 0 : max_rows;
+  }
+  const size_t total = static_cast<size_t>(n) * vec_per_row;
+  const size_t step = static_cast<size_t>(gridDim.x) * blockDim.x * kFlatBatch;
+  size_t base = static_cast<size_t>(blockIdx.x) * blockDim.x * kFlatBatch + threadIdx.x;
+  uint4 cur[kFlatBatch], nxt[kFlatBatch];
+#pragma unroll
+  for (int j = 0; j < kFlatBatch; ++j) {
+    const size_t i = base + static_cast<size_t>(j) * blockDim.x;
+    if (i < total) cur[j] = *flat_src(i, vec_per_row, V, ids, table, hot_rows, hot_slot, status, stats);
+  }
+  for (; base < total; base += step) {
+    const size_t nb = base + step;
+#pragma unroll
+    for (int j = 0; j < kFlatBatch; ++j) {
+      const size_t i = nb + static_cast<size_t>(j) * blockDim.x;
+      if (i < total) nxt[j] = *flat_src(i, vec_per_row, V, ids, table, hot_rows, hot_slot, status, stats);
+    }
+#pragma unroll
+    for (int j = 0; j < kFlatBatch; ++j) {
+      const size_t i = base + static_cast<size_t>(j) * blockDim.x;
+      if (i < total) dst[i] = cur[j];
+    }
+#pragma unroll
+    for (int j = 0; j < kFlatBatch; ++j) cur[j] = nxt[j];
+  }
+}
+
 __global__ void __launch_bounds__(kHostLinkThreads)
-writeback_rows_kernel(int vec_per_row, const uint4* __restrict__ rows,
+writeback_rows_kernel(int max_rows, int vec_per_row, const uint4* __restrict__ rows,
                       const int32_t* __restrict__ unique_ids, const int32_t* __restrict__ n_rows,
                       uint4* __restrict__ host_rows, int32_t* __restrict__ host_ids,
-                      int32_t* __restrict__ host_n) {
-  const int n = *n_rows;
+                      int32_t* __restrict__ host_n, int32_t* status) {
+  int n = *n_rows;
+  if (n > max_rows || n < 0) {   // clamped to what the host buffers hold, and reported
+    if (blockIdx.x == 0 && threadIdx.x == 0) report_error(status, STEM_ERR_COUNT_RANGE, n);
+    n = n < 0 ? 0 : max_rows;
+  }
   const size_t total = static_cast<size_t>(n) * vec_per_row;
   const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
   size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -101,9 +171,20 @@ cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int3
   int blocks = (max_rows + rows_per_cta - 1) / rows_per_cta;
   const int cap = table_on_host ? kHostLinkCtas : device_sm_count() * 8;
   if (blocks > cap) blocks = cap;
+  if (!table_on_host) {
+    // a device table: flat copy, as many CTAs as the largest possible count needs, up to 8 per SM
+    const size_t per_cta = static_cast<size_t>(kThreads) * kFlatBatch;
+    const size_t need = (static_cast<size_t>(max_rows) * vec + per_cta - 1) / per_cta;
+    const int grid = static_cast<int>(need < static_cast<size_t>(device_sm_count()) * 8 ? need : device_sm_count() * 8);
+    gather_rows_flat_kernel<<<grid > 0 ? grid : 1, kThreads, 0, stream>>>(
+        max_rows, V, vec, ids, n_ids, static_cast<const uint4*>(table), static_cast<const uint4*>(hot_rows), hot_slot,
+        static_cast<uint4*>(dst), status, stats);
+    count_launches(1);
+    return cudaGetLastError();
+  }
   static PerDeviceOnce configured;
   if (cudaError_t ce = configured.run([] { return prefer_max_shared(gather_rows_kernel); })) return ce;
-  gather_rows_kernel<<<blocks, threads, 0, stream>>>(V, vec, ids, n_ids, static_cast<const uint4*>(table),
+  gather_rows_kernel<<<blocks, threads, 0, stream>>>(max_rows, V, vec, ids, n_ids, static_cast<const uint4*>(table),
                                                     static_cast<const uint4*>(hot_rows), hot_slot,
                                                     static_cast<uint4*>(dst), status, stats);
   count_launches(1);
@@ -112,14 +193,14 @@ cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int3
 
 cudaError_t launch_writeback_rows(int max_rows, size_t row_bytes, const void* rows,
                                   const int32_t* unique_ids, const int32_t* n_rows, void* host_rows,
-                                  int32_t* host_ids, int32_t* host_n, cudaStream_t stream) {
+                                  int32_t* host_ids, int32_t* host_n, int32_t* status, cudaStream_t stream) {
   if (max_rows <= 0) return cudaSuccess;
   const int vec = static_cast<int>(row_bytes / 16);
   const int blocks = kHostLinkCtas;
   static PerDeviceOnce configured;
   if (cudaError_t ce = configured.run([] { return prefer_max_shared(writeback_rows_kernel); })) return ce;
-  writeback_rows_kernel<<<blocks, kHostLinkThreads, 0, stream>>>(vec, static_cast<const uint4*>(rows), unique_ids,
-                                                        n_rows, static_cast<uint4*>(host_rows), host_ids, host_n);
+  writeback_rows_kernel<<<blocks, kHostLinkThreads, 0, stream>>>(max_rows, vec, static_cast<const uint4*>(rows), unique_ids,
+                                                        n_rows, static_cast<uint4*>(host_rows), host_ids, host_n, status);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -5,11 +5,14 @@
 // (block, column slab) walks its positions in order, accumulating in fp32 registers.  A run
 // whose segment lies wholly inside the block is final and is written to dE_rows; a run whose
 // segment crosses a block edge (at most the first and the last run of a block) goes to a
-// partial row.  The CTAs that hold parts of such a segment count themselves off on an
-// integer counter; the one that arrives last adds the segment's partial rows in block order
-// and writes the row.  Which CTA that is varies from run to run, the order of the additions
-// does not, so the result is bitwise reproducible.  One launch; HBM-bound: every dU row is
-// read once with 16-byte loads, coalesced along d_ff.
+// partial row, and the block in which such a segment starts leaves a note (row, first and last
+// position).  A second, small kernel reads the notes and adds each crossing segment's partial
+// rows in block order.  No counters, no atomics, no state that outlives the call: the order of
+// every addition is fixed, so the result is bitwise reproducible.  Both kernels are launched
+// with programmatic stream serialisation and wait for the grid before them first, so they cost
+// no full launch boundary inside a chain of such kernels.  HBM-bound: every dU row is read once
+// with 16-byte loads, coalesced along d_ff.
+#include "ptx_sm100.cuh"
 #include "stem_internal.h"
 
 namespace stem {
@@ -19,6 +22,7 @@ constexpr int kSegBlk = 64;     // most sorted positions per CTA (the launch pic
 constexpr int kCtasPerSm = 7;   // register budget the kernel is compiled for
 constexpr int kThreads = 128;   // pass 1: one thread per vector of columns
 constexpr int kBatch = 8;       // rows requested before the first is consumed
+constexpr int kFinBatch = 8;    // finishing kernel: partial rows requested before the first is added
 
 template <typename T> struct Vec;
 template <> struct Vec<float> {
@@ -61,27 +65,29 @@ __device__ __forceinline__ void store_row(TOut* dst, const float (&v)[VI]) {
   for (int i = 0; i < VI; i += Vec<TOut>::N) Vec<TOut>::store(dst + i, v + i);
 }
 
-// Scratch layout: arrival counters [n_blk][n_slabs] (one per block in which a crossing
-// segment can start, per column slab; zeroed before each launch), then 2 partial rows per
-// block.
-__host__ __device__ inline size_t partial_offset_bytes(int n_blk, int n_slabs) {
-  return (static_cast<size_t>(n_blk) * n_slabs * 4 + 255) / 256 * 256;
+// Scratch layout: one note per block (int4: row of the crossing segment that starts in the
+// block or -1, its first position, its end position, unused; written by the block's CTA of
+// column slab 0 on every launch), then 2 partial rows per block.
+__host__ __device__ inline size_t partial_offset_bytes(int n_blk) {
+  return (static_cast<size_t>(n_blk) * sizeof(int4) + 255) / 256 * 256;
 }
 
 template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 segreduce_kernel(int T, int F, int blk_len, const TIn* __restrict__ dU, const int32_t* __restrict__ perm,
                  const int32_t* __restrict__ seg_offsets, const int32_t* __restrict__ n_unique,
-                 TOut* __restrict__ dE_rows, int32_t* __restrict__ counters, float* partial) {
+                 TOut* __restrict__ dE_rows, int4* __restrict__ notes, float* partial) {
   constexpr int VI = (Vec<TIn>::N > Vec<TOut>::N) ? Vec<TIn>::N : Vec<TOut>::N;
   constexpr int LD = VI / Vec<TIn>::N;  // 16-byte loads per row per thread
   __shared__ int s_off[kSegBlk + 1];    // offsets of the segments that can touch this block
   __shared__ int s_row[kSegBlk];
   __shared__ int s_loc[kSegBlk];        // position -> index into s_off
-  __shared__ int s_finish[2];           // crossing segments this CTA must finish (index into s_off), or -1
   const int blk = blockIdx.x;
   const int p0 = blk * blk_len;
   const int cnt = min(blk_len, T - p0);
+  // everything below reads what earlier kernels of the stream produced
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
   const int n_u = *n_unique;
 
   // r_first = largest r with seg_offsets[r] <= p0, found with kThreads pivots per round
@@ -154,49 +160,71 @@ segreduce_kernel(int T, int F, int blk_len, const TIn* __restrict__ dU, const in
     }
   }
 
-  // ---- crossing segments: the last CTA to arrive adds the parts ----------------------------
-  // At most two per block: the segment of the first position (if it began earlier or runs on)
-  // and that of the last position (if it runs on).  s_off[0] <= p0, so index 0 is the first.
-  __threadfence();   // this CTA's partial rows are visible before it counts itself off
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int n_slabs = gridDim.y;
-    const int j_first = 0, j_last = s_loc[cnt - 1];
-    for (int which = 0; which < 2; ++which) {
-      const int j = which == 0 ? j_first : j_last;
-      int fin = -1;
-      const bool whole = s_off[j] >= p0 && s_off[j + 1] <= p0 + blk_len;
-      if (!whole && !(which == 1 && j_last == j_first)) {
-        const int start_blk = s_off[j] / blk_len, last_blk = (s_off[j + 1] - 1) / blk_len;
-        const int old = atomicAdd(&counters[start_blk * n_slabs + blockIdx.y], 1);
-        if (old == last_blk - start_blk) fin = j;
-      }
-      s_finish[which] = fin;
-    }
+  // ---- the note for the finishing kernel: the crossing segment that starts in this block ------
+  // Only the segment of the block's last position can start here and run on.  s_off[0] <= p0.
+  if (blockIdx.y == 0 && threadIdx.x == 0) {
+    const int j = s_loc[cnt - 1];
+    const bool starts_here = s_off[j] >= p0, runs_on = s_off[j + 1] > p0 + blk_len;
+    notes[blk] = (starts_here && runs_on) ? make_int4(r_first + j, s_off[j], s_off[j + 1], 0) : make_int4(-1, 0, 0, 0);
   }
-  __syncthreads();
+}
+
+// Finishing kernel: one CTA per (block, column slab).  If a crossing segment starts in the block,
+// add its partial rows in block order and write the row.
+template <typename TOut>
+__global__ void __launch_bounds__(kThreads)
+segfinish_kernel(int F, int blk_len, int vi, const int4* __restrict__ notes, const float* __restrict__ partial,
+                 TOut* __restrict__ dE_rows) {
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
+  const int4 note = __ldcg(notes + blockIdx.x);
+  if (note.x < 0) return;
+  const int seg_begin = note.y, seg_end = note.z;
+  const int start_blk = blockIdx.x, last_blk = (seg_end - 1) / blk_len;
+  // the same columns per thread as in the first kernel: vi consecutive columns, in groups of 4
+  const int col0 = (blockIdx.y * kThreads + threadIdx.x) * vi;
+  if (col0 >= F) return;
+  for (int c = 0; c < vi; c += 4) {
+    const int col = col0 + c;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    // parts are requested kFinBatch at a time and added in block order: a segment of a frequent id
+    // spans dozens of blocks, and one load latency per block would make this launch a serial tail
+    for (int b0 = start_blk; b0 <= last_blk; b0 += kFinBatch) {
+      float4 q[kFinBatch];
 #pragma unroll
-  for (int which = 0; which < 2; ++which) {
-    const int j = s_finish[which];
-    if (j < 0 || !col_ok) continue;
-    __threadfence();   // the other CTAs' partial rows, published before their count, are visible
-    const int seg_begin = s_off[j], seg_end = s_off[j + 1];
-    const int start_blk = seg_begin / blk_len, last_blk = (seg_end - 1) / blk_len;
+      for (int i = 0; i < kFinBatch; ++i) {
+        const int b = b0 + i;
+        if (b <= last_blk) {
+          // the segment's run is the first run of block b, unless b is the block it starts in
+          // and it does not start at that block's first position
+          const int slot = (b > start_blk || seg_begin == start_blk * blk_len) ? 2 * b : 2 * b + 1;
+          q[i] = __ldcg(reinterpret_cast<const float4*>(partial + static_cast<size_t>(slot) * F + col));
+        }
+      }
 #pragma unroll
-    for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
-    for (int b = start_blk; b <= last_blk; ++b) {
-      // the segment's run is the first run of block b, unless b is the block it starts in
-      // and it does not start at that block's first position
-      const int slot = (b > start_blk || seg_begin == start_blk * blk_len) ? 2 * b : 2 * b + 1;
-      const float* src = partial + static_cast<size_t>(slot) * F + col;
-#pragma unroll
-      for (int i = 0; i < VI; i += 4) {
-        const float4 q = __ldcg(reinterpret_cast<const float4*>(src + i));
-        acc[i] += q.x; acc[i + 1] += q.y; acc[i + 2] += q.z; acc[i + 3] += q.w;
+      for (int i = 0; i < kFinBatch; ++i) {
+        if (b0 + i <= last_blk) { acc.x += q[i].x; acc.y += q[i].y; acc.z += q[i].z; acc.w += q[i].w; }
       }
     }
-    store_row<VI, TOut>(dE_rows + static_cast<size_t>(r_first + j) * F + col, acc);
+    TOut* dst = dE_rows + static_cast<size_t>(note.x) * F + col;
+    dst[0] = from_f32<TOut>(acc.x); dst[1] = from_f32<TOut>(acc.y);
+    dst[2] = from_f32<TOut>(acc.z); dst[3] = from_f32<TOut>(acc.w);
   }
+}
+
+// Resident CTAs of the first kernel per SM, per device (an occupancy query is not free).
+template <typename TIn, typename TOut>
+int ctas_per_sm() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, segreduce_kernel<TIn, TOut>, kThreads, 0) != cudaSuccess || n < 1)
+      n = 1;
+    cached[dev] = n;
+  }
+  return cached[dev];
 }
 
 template <typename TIn, typename TOut>
@@ -207,28 +235,33 @@ cudaError_t launch_typed(int T, int F, const void* dU, const int32_t* perm, cons
   // Block length: as long as allowed, then shortened so that the CTAs fill a whole number of
   // waves of the resident CTA slots (a ragged last wave of full-length blocks costs more than
   // evenly shorter blocks).
-  static int ctas_per_sm = 0;
-  if (ctas_per_sm == 0) {
-    int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, segreduce_kernel<TIn, TOut>, kThreads, 0) != cudaSuccess || n < 1)
-      n = 1;
-    ctas_per_sm = n;
-  }
-  const int per_wave = device_sm_count() * ctas_per_sm / n_slabs > 0 ? device_sm_count() * ctas_per_sm / n_slabs : 1;
+  const int resident = ctas_per_sm<TIn, TOut>();
+  const int per_wave = device_sm_count() * resident / n_slabs > 0 ? device_sm_count() * resident / n_slabs : 1;
   const int min_blk = (T + kSegBlk - 1) / kSegBlk;
   const int waves = (min_blk + per_wave - 1) / per_wave;
   int blk_len = (T + waves * per_wave - 1) / (waves * per_wave);
   if (blk_len < 8) blk_len = 8 < T ? 8 : T;
   if (blk_len > kSegBlk) blk_len = kSegBlk;
   const int n_blk = (T + blk_len - 1) / blk_len;
-  int32_t* counters = static_cast<int32_t*>(scratch);
-  float* partial = reinterpret_cast<float*>(static_cast<char*>(scratch) + partial_offset_bytes(n_blk, n_slabs));
-  cudaError_t e = cudaMemsetAsync(counters, 0, static_cast<size_t>(n_blk) * n_slabs * sizeof(int32_t), stream);
-  if (e != cudaSuccess) return e;
-  segreduce_kernel<TIn, TOut><<<dim3(n_blk, n_slabs), kThreads, 0, stream>>>(
-      T, F, blk_len, static_cast<const TIn*>(dU), perm, seg_offsets, n_unique, static_cast<TOut*>(dE_rows), counters, partial);
+  int4* notes = static_cast<int4*>(scratch);
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(scratch) + partial_offset_bytes(n_blk));
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_blk, n_slabs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, segreduce_kernel<TIn, TOut>, T, F, blk_len, static_cast<const TIn*>(dU), perm,
+                                     seg_offsets, n_unique, static_cast<TOut*>(dE_rows), notes, partial);
   count_launches(1);
-  return cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  e = cudaLaunchKernelEx(&cfg, segfinish_kernel<TOut>, F, blk_len, VI, static_cast<const int4*>(notes),
+                         static_cast<const float*>(partial), static_cast<TOut*>(dE_rows));
+  count_launches(1);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
@@ -237,8 +270,7 @@ size_t segreduce_workspace_bytes(int T, int F) {
   if (T <= 0) return 0;
   // bounds over every launch shape: blocks of at least 8 positions, the narrowest slab
   const size_t n_blk = (static_cast<size_t>(T) + 7) / 8;
-  const int n_slabs = (F + kThreads * 4 - 1) / (kThreads * 4);
-  return partial_offset_bytes(static_cast<int>(n_blk), n_slabs) + align_up(2 * n_blk * static_cast<size_t>(F) * sizeof(float), 256);
+  return partial_offset_bytes(static_cast<int>(n_blk)) + align_up(2 * n_blk * static_cast<size_t>(F) * sizeof(float), 256);
 }
 
 cudaError_t launch_segreduce(int T, int F, int in_dtype, int out_dtype, const void* dU,

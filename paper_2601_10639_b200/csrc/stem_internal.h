@@ -74,6 +74,15 @@ cudaError_t launch_simt_gemm(int dtype, int M, int N, int K, const void* A, bool
 cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const void* B,
                            bool b_mn, EpiKind kind, const EpiParams& ep, bool pair, cudaStream_t stream);
 
+// Two token-contracted products in one launch (the two weight gradients of the layer):
+//   out1[m,n] = sum_k A1(k,m) B1(k,n)   and   out2[m,n] = sum_k A2(k,m) B2(k,n),
+// all four operands stored [K, .] row-major (MN-major), both outputs of ep.out_fp32's type, the
+// same ep.accumulate.  Their tiles share one work list, so the pair fills the SMs where each
+// product alone leaves some idle; ep.out is ignored (out1 / out2 are the outputs).
+cudaError_t launch_tc_gemm_token_pair(int K, int M1, int N1, const void* A1, const void* B1, void* out1, int M2,
+                                      int N2, const void* A2, const void* B2, void* out2, const EpiParams& ep,
+                                      bool pair, cudaStream_t stream);
+
 size_t tc_gemm_scratch_bytes();
 
 // ---- index path ----------------------------------------------------------------------
@@ -103,7 +112,7 @@ cudaError_t launch_gather_rows(int max_rows, int V, size_t row_bytes, const int3
                                int32_t* stats, cudaStream_t stream);
 cudaError_t launch_writeback_rows(int max_rows, size_t row_bytes, const void* rows,
                                   const int32_t* unique_ids, const int32_t* n_rows, void* host_rows,
-                                  int32_t* host_ids, int32_t* host_n, cudaStream_t stream);
+                                  int32_t* host_ids, int32_t* host_n, int32_t* status, cudaStream_t stream);
 
 // ---- frequency-ranked row cache ------------------------------------------------------------
 size_t lfu_workspace_bytes(int V, int K);
@@ -119,6 +128,10 @@ cudaError_t launch_shard_route(int n_max, int T, int G, const int32_t* unique_id
                                const int32_t* inverse, int32_t* send_local, int32_t* send_slot,
                                int32_t* send_counts, int32_t* token_slot, void* scratch, int32_t* status,
                                cudaStream_t stream);
+
+// Bounded-wait self-test (selftest.cu): one thread waits at most limit_cycles on a barrier that
+// is completed first (arrive != 0) or never.
+cudaError_t launch_selftest_wait(int32_t* status, long long limit_cycles, int arrive, cudaStream_t stream);
 
 int device_sm_count();
 

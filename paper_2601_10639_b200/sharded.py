@@ -54,6 +54,27 @@ class DistExchange:
         self.dist.all_to_all_single(out, inp, group=self.group)
         return [int(v) for v in out.tolist()]
 
+    def counts_from_device(self, send_counts_dev: torch.Tensor) -> Tuple[List[int], List[int]]:
+        """The same exchange starting from the device-resident request counts (int32 [G], as
+        stem_shard_route leaves them): the all-to-all runs on them where they are, and both
+        lists -- what this rank sends to each owner, what it receives from each requester -- reach
+        the host in ONE copy, the only host round trip of a step (the sizes of the variable-length
+        exchanges have to be known on the host)."""
+        nccl = self.dist.get_backend(self.group) == "nccl"
+        inp = send_counts_dev if nccl else send_counts_dev.cpu()
+        both = torch.empty(2, self.G, dtype=inp.dtype, device=inp.device)
+        both[0].copy_(inp)
+        self.dist.all_to_all_single(both[1], both[0], group=self.group)
+        if nccl:
+            if getattr(self, "_pinned", None) is None:
+                self._pinned = torch.empty(2, self.G, dtype=inp.dtype).pin_memory()
+            self._pinned.copy_(both, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            host = self._pinned
+        else:
+            host = both
+        return [int(v) for v in host[0].tolist()], [int(v) for v in host[1].tolist()]
+
     def rows(self, send: torch.Tensor, send_counts: Sequence[int], recv_counts: Sequence[int]) -> torch.Tensor:
         recv = torch.empty((sum(recv_counts),) + tuple(send.shape[1:]), dtype=send.dtype, device=send.device)
         self.dist.all_to_all_single(recv, send[:sum(send_counts)].contiguous(), list(recv_counts), list(send_counts),
@@ -105,14 +126,15 @@ class ShardedRank:
         self.recv_local = None
 
     # -- A: dedup + route ----------------------------------------------------------------
-    def phase_route(self, x, ids, dy) -> List[int]:
+    def phase_route(self, x, ids, dy, read_counts: bool = True) -> List[int]:
         L = self.layer
         L.x, L.ids, L.dy = x, ids, dy
         L.dedup()
         b = L.bufs
         B.stem_shard_route(self.n_max, self.shape.T, self.G, b["unique_ids"], b["n_unique"], b["inverse"],
                            self.send_local, self.send_slot, self.send_counts, self.token_slot, self.route_ws)
-        self.h_send_counts = [int(v) for v in self.send_counts.tolist()]   # sizes the exchange (host round trip)
+        if read_counts:     # sizes the exchange (host round trip); step_dist reads them with the peers' counts instead
+            self.h_send_counts = [int(v) for v in self.send_counts.tolist()]
         return self.h_send_counts
 
     # -- B: owner side of the forward exchange -------------------------------------------------
@@ -185,16 +207,21 @@ class ShardedRank:
         return st if st != B.OK or ob is None else B.stem_query_status(ob["ws"])
 
     # -- one step, one process per GPU ---------------------------------------------------------
-    def step_dist(self, ex: DistExchange, x, ids, dy):
-        send_counts = self.phase_route(x, ids, dy)
-        recv_counts = ex.counts(send_counts, self.device)
+    def step_dist(self, ex: DistExchange, x, ids, dy, timed=None):
+        """One step of this rank among ex.G processes.  `timed(name, fn)` may wrap each phase (the
+        benchmark brackets them with CUDA events): route, counts, serve, layer, reduce and the three
+        row exchanges x_ids, x_rows, x_grads."""
+        run = timed or (lambda name, fn: fn())
+        run("route", lambda: self.phase_route(x, ids, dy, read_counts=False))
+        send_counts, recv_counts = run("counts", lambda: ex.counts_from_device(self.send_counts))
+        self.h_send_counts = send_counts
         n_u = sum(send_counts)
-        recv_local = ex.rows(self.send_local[:n_u], send_counts, recv_counts)
-        served = self.phase_serve(recv_local, recv_counts)
-        rows = ex.rows(served, recv_counts, send_counts)
-        grads = self.phase_layer(rows)
-        recv_grads = ex.rows(grads, send_counts, recv_counts)
-        return self.phase_reduce(recv_grads)
+        recv_local = run("x_ids", lambda: ex.rows(self.send_local[:n_u], send_counts, recv_counts))
+        served = run("serve", lambda: self.phase_serve(recv_local, recv_counts))
+        rows = run("x_rows", lambda: ex.rows(served, recv_counts, send_counts))
+        grads = run("layer", lambda: self.phase_layer(rows))
+        recv_grads = run("x_grads", lambda: ex.rows(grads, send_counts, recv_counts))
+        return run("reduce", lambda: self.phase_reduce(recv_grads))
 
 
 def step_local(ranks: List[ShardedRank], ex: LocalExchange, xs, idss, dys, timed=None):

@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_version_and_status_strings():
     assert B.stem_version() >= 100
-    for code in range(0, -9, -1):
+    for code in range(0, -11, -1):
         s = B.status_string(code)
         assert s and s != "unknown status"
     assert B.status_string(-99) == "unknown status"
@@ -109,8 +109,11 @@ def test_later_entry_points_reject_bad_arguments_on_the_host():
     args = [ctypes.byref(s)] + [None] * 15 + [0, None]
     assert L.stem_ffn_step_host(*args) == B.ERR_INVALID_ARG
     assert L.stem_step_arena_bytes(ctypes.byref(s), ctypes.byref(sz)) == B.OK and sz.value > 0
-    for code in (B.OK, B.ERR_STATIC_LIMIT):
+    for code in (B.OK, B.ERR_STATIC_LIMIT, B.ERR_COUNT_RANGE):
         assert B.status_string(code)
+    assert L.stem_selftest_wait(None, 1000, 0, None) == B.ERR_INVALID_ARG
+    assert L.stem_selftest_wait(0x1000, 0, 0, None) == B.ERR_INVALID_ARG                      # limit below 1
+    assert L.stem_selftest_wait(0x1000, 3000000000, 0, None) == B.ERR_INVALID_ARG             # limit above 2e9
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
