@@ -58,7 +58,11 @@ def load_peaks():
     if os.path.exists(p):
         with open(p) as f:
             d = json.load(f)
-        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+        out = {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+        under = (d.get("clocks_under_load") or {}).get("sm_mhz_median")
+        if under:
+            out["sm_mhz_under_load"] = float(under)
+        return out
     return dict(FALLBACK_PEAKS, source="fallback")
 
 
@@ -102,7 +106,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -648,6 +652,299 @@ def run_sharded(args, w):
     }))
 
 
+NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}   # dense bf16 and HBM3e figures of the data sheet
+
+
+def roofline_regime(region_s: float, sm_mhz, peaks) -> str:
+    """Which measured tensor peak a timed region is compared with: the burst figure when the region
+    is too short to settle under the power cap (under a second) or ran at clocks well above those
+    the sustained figure was measured at, else the sustained one."""
+    under_load = peaks.get("sm_mhz_under_load")
+    if region_s < 1.0:
+        return "burst"
+    if sm_mhz and under_load and sm_mhz > 1.15 * under_load:
+        return "burst"
+    return "sustained"
+
+
+def measure_layer(w, T, steps, warmup, args, rank, local, dev, barrier, variant, profile=True):
+    """Device-resident timing of dedup + forward (+ backward) of one layer: synthetic inputs made on
+    the device, `warmup` untimed steps, `steps` timed ones between two CUDA events, per-step-of-the-
+    path event records, clocks sampled meanwhile."""
+    import torch
+    from paper_2601_10639_b200 import binding as B
+    from paper_2601_10639_b200 import runner
+
+    dcode = B.DTYPE_BF16 if w.dtype == "bf16" else B.DTYPE_FP32
+    dt = runner.torch_dtype(dcode)
+    d, F, V, backward = w.d_model, w.d_ff, w.V, w.backward
+    gen = torch.Generator(device=dev).manual_seed(args.seed + 1000 * rank)
+    st = runner.LayerState(B.make_shape(T, d, F, V, dcode, B.DTYPE_FP32, 0), device=dev)
+    st.x = torch.randn(T, d, generator=gen, device=dev, dtype=torch.float32).to(dt)
+    st.dy = torch.randn(T, d, generator=gen, device=dev, dtype=torch.float32).to(dt)
+    st.W_gate = (torch.randn(F, d, generator=gen, device=dev, dtype=torch.float32) * d ** -0.5).to(dt)
+    st.W_down = (torch.randn(d, F, generator=gen, device=dev, dtype=torch.float32) * F ** -0.5).to(dt)
+    st.E = torch.empty(V, F, device=dev, dtype=dt)
+    for r0 in range(0, V, 4096):
+        r1 = min(V, r0 + 4096)
+        st.E[r0:r1] = (torch.randn(r1 - r0, F, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(dt)
+    ids_np = synth.token_ids(rank_seed(args.seed, rank), T, V, w.id_dist)
+    st.ids = torch.from_numpy(ids_np).to(dev)
+    st.allocate(backward)
+    stream = torch.cuda.current_stream()
+    run_step = lambda: st.step(backward=backward)
+    if variant == "dagger":
+        # STEM-dagger (Appendix): the up-projection is kept; 3 contractions forward, 6 backward
+        W_up = (torch.randn(F, d, generator=gen, device=dev, dtype=torch.float32) * d ** -0.5).to(dt)
+        U = torch.empty(T, F, dtype=dt, device=dev)
+        dW_up = torch.empty(F, d, dtype=torch.float32, device=dev)
+        b_ = st.bufs
+
+        def run_step():
+            st.dedup()
+            B.stem_dagger_forward(st.shape, st.x, st.ids, st.W_gate, W_up, st.E, st.W_down, b_["y"], b_["G"], b_["H"], U,
+                                  b_["ws"])
+            if backward:
+                B.stem_dagger_backward(st.shape, st.dy, st.x, st.W_gate, W_up, st.W_down, b_["G"], b_["H"], U, b_["perm"],
+                                       b_["seg_offsets"], b_["n_unique"], b_["dx"], b_["dW_gate"], dW_up, b_["dW_down"],
+                                       b_["dE_rows"], b_["ws"])
+
+    for _ in range(warmup):
+        run_step()
+    barrier()
+    assert st.status() == B.OK, B.status_string(st.status())
+    n_u = int(st.bufs["n_unique"].item())
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = B.stem_launch_count()
+    with ClockSampler(local) as clocks:
+        B.stem_profile_enable(profile)
+        barrier()
+        t0 = time.time()
+        ev0.record(stream)
+        for _ in range(steps):
+            run_step()
+        ev1.record(stream)
+        barrier()
+        t1 = time.time()
+        B.stem_profile_enable(False)
+    launches = B.stem_launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    records = B.stem_profile_records()
+    assert st.status() == B.OK, B.status_string(st.status())
+    return {"state": st, "n_unique": n_u, "ids_np": ids_np, "dcode": dcode, "ms_total": ms_total, "records": records,
+            "launches": launches, "clocks": clocks.summary(t0, t1)}
+
+
+def measure_gather(st, n_u, T, V, F, esz, dev):
+    """cache[r] = E[unique_ids[r]] on the device, back to back, outside the timed step."""
+    import torch
+    from paper_2601_10639_b200 import binding as B
+    cache = torch.empty(min(T, V), F, dtype=st.E.dtype, device=dev)
+    b = st.bufs
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        B.stem_prefetch_rows(st.shape, b["unique_ids"], b["n_unique"], st.E, cache, b["ws"])
+    torch.cuda.synchronize()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 20
+    g0.record(stream)
+    for _ in range(reps):
+        B.stem_prefetch_rows(st.shape, b["unique_ids"], b["n_unique"], st.E, cache, b["ws"])
+    g1.record(stream)
+    torch.cuda.synchronize()
+    return {"rows": n_u, "ms": g0.elapsed_time(g1) / reps, "bytes": 2 * n_u * F * esz}     # rows read once, written once
+
+
+def gather_entry(gather, peaks):
+    gbs = gather["bytes"] / (gather["ms"] * 1e-3) / 1e9
+    return {"launch_sets": 20, "avg_ms": gather["ms"], "rows": gather["rows"], "bytes": gather["bytes"], "gbs": gbs,
+            "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_hbm": gbs / NOMINAL["hbm_gbs"],
+            "note": "cache[r] = E[unique_ids[r]] on the device, back to back, outside the timed step"}
+
+
+def kernel_table(records, ms_total, T, d, F, n_u, esz, grad_fp32, peaks):
+    """Per step of the path: average event time, share of the timed region, and the achieved rate
+    against the measured (burst and sustained) and nominal peaks."""
+    by_name: dict[str, list] = {}
+    for name, ms in records:
+        by_name.setdefault(name, []).append(ms)
+    flops_gemm = 2.0 * T * d * F
+    seg_bytes = T * F * esz + n_u * F * (4 if grad_fp32 else 2) + 4 * (T + n_u + 1)
+    kernels = {}
+    for name, v in by_name.items():
+        avg = float(np.mean(v))
+        k = {"launch_sets": len(v), "avg_ms": avg, "share": float(np.sum(v)) / ms_total}
+        if name.endswith("_gemm"):
+            # the two weight gradients run as one launch: twice the work of one contraction
+            k["tflops"] = (2.0 if name == "dw_pair_gemm" else 1.0) * flops_gemm / (avg * 1e-3) / 1e12
+            k["frac_of_measured_sustained"] = k["tflops"] / peaks["bf16_tflops_sustained"]
+            k["frac_of_measured_burst"] = k["tflops"] / peaks["bf16_tflops"]
+            k["frac_of_nominal"] = k["tflops"] / NOMINAL["bf16_tflops"]
+        elif name == "seg_reduce":
+            k["bytes"] = seg_bytes
+            k["gbs"] = seg_bytes / (avg * 1e-3) / 1e9
+            k["frac_of_measured_hbm"] = k["gbs"] / peaks["hbm_gbs"]
+            k["frac_of_nominal_hbm"] = k["gbs"] / NOMINAL["hbm_gbs"]
+        kernels[name] = k
+    return kernels
+
+
+def rooflines(kernels, regime, peaks, T, d, F, bf16):
+    """The two roofline objects of a bench line: the slowest contraction against the measured tensor
+    peak of the run's regime, and the slower of the two HBM-bound kernels against the measured copy
+    bandwidth."""
+    gemms = {n: k for n, k in kernels.items() if n.endswith("_gemm")}
+    roofline = None
+    if gemms and bf16:
+        dom = min(gemms, key=lambda n: gemms[n]["tflops"])      # the contraction furthest from the peak
+        cap = load_traffic(dom)
+        # DRAM traffic grows in proportion to the tokens of a launch (every [T,.] operand does; the
+        # weights are the small remainder), so a capture at fewer tokens is scaled by T / T_captured.
+        traffic = cap[1] * T / cap[0] if cap else None
+        key = "bf16_tflops" if regime == "burst" else "bf16_tflops_sustained"
+        g = gemms[dom]
+        roofline = {"kernel": dom, "bound": "tensor", "achieved": g["tflops"], "peak": peaks[key], "unit": "TFLOP/s",
+                    "frac": g["tflops"] / peaks[key], "regime": regime,
+                    "frac_burst": g["frac_of_measured_burst"], "frac_sustained": g["frac_of_measured_sustained"],
+                    "frac_nominal": g["frac_of_nominal"], "traffic": traffic,
+                    "peak_source": f"{peaks['source']} ({regime} bf16 GEMM, of measured); nominal 2250 TFLOP/s",
+                    "flops_per_launch": (2.0 if dom == "dw_pair_gemm" else 1.0) * 2.0 * T * d * F}
+    hbm = {n: k for n, k in kernels.items() if "frac_of_measured_hbm" in k}
+    roofline_hbm = None
+    if hbm:
+        worst = min(hbm, key=lambda n: hbm[n]["frac_of_measured_hbm"])
+        k = hbm[worst]
+        roofline_hbm = {"kernel": worst, "bound": "hbm", "achieved": k["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": k["frac_of_measured_hbm"], "frac_nominal": k["frac_of_nominal_hbm"],
+                        "bytes_per_launch": k["bytes"], "traffic": None,
+                        "peak_source": f"{peaks['source']} (copy bandwidth, of measured); nominal 8000 GB/s",
+                        "all": {n: v["frac_of_measured_hbm"] for n, v in hbm.items()}}
+    return roofline, roofline_hbm
+
+
+def shard_plan(V: int, world: int, rank: int) -> dict:
+    """Which rows of a V-row table rank `rank` of `world` holds (row id lives on rank id mod world at
+    local index id // world) and how a batch's distinct ids spread over the owners on average."""
+    from paper_2601_10639_b200 import sharded
+    return {"rank": rank, "world": world, "rows_owned": sharded.shard_rows(V, world, rank),
+            "first_id": rank, "id_stride": world}
+
+
+def sharded_line(args, w, T, world, ms_total, phase_ms, plan, sent, launches, clocks) -> dict:
+    """The JSON line of the sharded mode from rank 0's view: times are maxima over ranks already."""
+    F = w.d_ff
+    n_u, remote = sum(sent), sum(c for g, c in enumerate(sent) if g != plan["rank"])
+    ms_per_step = ms_total / args.steps
+    return {
+        "metric": "STEM-FFN fwd+bwd tokens/sec with the table sharded over the GPUs (id mod N), replicated weights",
+        "value": world * T * args.steps / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "T": T, "d_model": w.d_model, "d_ff": F, "V": w.V, "ids": w.id_dist,
+                   "parallelism": f"table sharded id mod {world} + replicas x{world}", "exchange": "NCCL all-to-all-v",
+                   "rows_owned_rank0": plan["rows_owned"],
+                   "l2": "per-step working set exceeds the 126 MB L2; no flush"},
+        "gpu_launches": int(launches), "clocks": clocks,
+        "tflops_step": world * layer_flops(T, w.d_model, F, True) / (ms_per_step * 1e-3) / 1e12,
+        "ms_per_phase_max_over_ranks": phase_ms,
+        "rank0_rows": {"distinct": n_u, "from_other_ranks": remote},
+        "rank0_exchange_bytes": {"ids_out": 4 * remote, "rows_in": remote * F * 2, "grad_rows_out_fp32": remote * F * 4},
+        "host_round_trips_per_step": 1,
+    }
+
+
+def run_sharded_dist(args, w):
+    """The layer with its table sharded over the ranks of a torch.distributed job (paper Section 3.4,
+    "parallel embeddings"): one process per GPU, rows and gradient rows exchanged by NCCL all-to-all-v,
+    every rank its own batch.  A step = route, exchange, forward, backward, exchange, the owner's
+    reduce.  Times are CUDA-event times, maximum over ranks; rank 0 prints the line."""
+    import socket
+    import torch
+    import torch.distributed as dist
+    from paper_2601_10639_b200 import binding as B
+    from paper_2601_10639_b200 import sharded
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    os.environ.setdefault("NCCL_DEBUG", "INFO")               # keep the communicator's own log (stderr)
+    os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    if "MASTER_ADDR" not in os.environ:                       # a plain `python bench.py --sharded`: a group of one
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    B.lib()
+    dt = torch.bfloat16
+    T, d, F, V = (args.tokens or w.T), w.d_model, w.d_ff, w.V
+    plan = shard_plan(V, world, rank)
+    shape = B.make_shape(T, d, F, V, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    gen = torch.Generator(device=dev).manual_seed(args.seed)         # weights and table: the same on every rank
+    W_gate = (torch.randn(F, d, generator=gen, device=dev) * d ** -0.5).to(dt)
+    W_down = (torch.randn(d, F, generator=gen, device=dev) * F ** -0.5).to(dt)
+    shard = torch.empty(plan["rows_owned"], F, device=dev, dtype=dt)
+    for r0 in range(0, V, 4096):                                     # the whole table is drawn, this rank keeps its rows
+        r1 = min(V, r0 + 4096)
+        blk = (torch.randn(r1 - r0, F, generator=gen, device=dev) * 0.02).to(dt)
+        first = (rank - r0) % world                                   # first row of the block with id mod world == rank
+        mine = blk[first::world]
+        lo = (r0 + first) // world
+        shard[lo:lo + mine.shape[0]] = mine
+    gen_r = torch.Generator(device=dev).manual_seed(args.seed + 1000 * (rank + 1))    # the batch: every rank its own
+    x = torch.randn(T, d, generator=gen_r, device=dev).to(dt)
+    dy = torch.randn(T, d, generator=gen_r, device=dev).to(dt)
+    ids = torch.from_numpy(synth.token_ids(rank_seed(args.seed, rank), T, V, w.id_dist)).to(dev)
+    rk = sharded.ShardedRank(rank, world, shape, shard, W_gate, W_down, device=dev)
+    ex = sharded.DistExchange()
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        rk.step_dist(ex, x, ids, dy)
+    barrier()
+    assert rk.status() == B.OK
+    events = []
+
+    def timed(name, fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        out = fn()
+        e1.record(stream)
+        events.append((name, e0, e1))
+        return out
+
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = B.stem_launch_count()
+    with ClockSampler(local) as clocks:
+        barrier()
+        t0 = time.time()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            rk.step_dist(ex, x, ids, dy, timed)
+        ev1.record(stream)
+        barrier()
+        t1 = time.time()
+    launches = B.stem_launch_count() - launches0
+    assert rk.status() == B.OK
+    names = ["route", "counts", "x_ids", "serve", "x_rows", "layer", "x_grads", "reduce"]
+    sums = {n: 0.0 for n in names}
+    for name, e0, e1 in events:
+        sums[name] += e0.elapsed_time(e1) / args.steps
+    t = max_over_ranks([ev0.elapsed_time(ev1)] + [sums[n] for n in names], dev)
+    if rank == 0:
+        print(json.dumps(sharded_line(args, w, T, world, t[0], dict(zip(names, t[1:])), plan, rk.h_send_counts, launches,
+                                      clocks.summary(t0, t1))))
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -669,6 +966,10 @@ def main():
     ap.add_argument("--no-profile", action="store_true",
                     help="do not record per-step events inside the timed region (checks what they cost)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="default workload only: skip the short timings of the other single-layer configurations")
+    ap.add_argument("--sharded", action="store_true",
+                    help="the table sharded over the --gpus ranks of this job (one process per GPU, NCCL all-to-all-v)")
     ap.add_argument("--shard-ranks", type=int, default=0,
                     help="G > 0: the table sharded over G virtual ranks on one GPU (per-rank device times)")
     args = ap.parse_args()
@@ -683,6 +984,11 @@ def main():
         run_unique_growth(args)
         return
 
+    if args.sharded:
+        if w.host_tables or not w.backward or w.dtype != "bf16":
+            raise SystemExit("--sharded runs the single-layer bf16 training workloads")
+        run_sharded_dist(args, w)
+        return
     if args.shard_ranks > 0:
         if int(os.environ.get("WORLD_SIZE", "1")) > 1:
             raise SystemExit("--shard-ranks steps virtual ranks on one GPU")
@@ -702,7 +1008,6 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2601_10639_b200 import binding as B
-    from paper_2601_10639_b200 import runner
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -715,76 +1020,21 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     B.lib()  # fail loudly here if the extension is missing
 
-    dcode = B.DTYPE_BF16 if w.dtype == "bf16" else B.DTYPE_FP32
-    dt = runner.torch_dtype(dcode)
-    T, d, F, V = (args.tokens or w.T), w.d_model, w.d_ff, w.V
-    backward = w.backward
-    # ---- synthetic inputs (every rank its own batch; same shapes) -----------------------
-    gen = torch.Generator(device=dev).manual_seed(args.seed + 1000 * rank)
-    st = runner.LayerState(B.make_shape(T, d, F, V, dcode, B.DTYPE_FP32, 0), device=dev)
-    st.x = torch.randn(T, d, generator=gen, device=dev, dtype=torch.float32).to(dt)
-    st.dy = torch.randn(T, d, generator=gen, device=dev, dtype=torch.float32).to(dt)
-    st.W_gate = (torch.randn(F, d, generator=gen, device=dev, dtype=torch.float32) * d ** -0.5).to(dt)
-    st.W_down = (torch.randn(d, F, generator=gen, device=dev, dtype=torch.float32) * F ** -0.5).to(dt)
-    st.E = torch.empty(V, F, device=dev, dtype=dt)
-    for r0 in range(0, V, 4096):
-        r1 = min(V, r0 + 4096)
-        st.E[r0:r1] = (torch.randn(r1 - r0, F, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(dt)
-    ids_np = synth.token_ids(rank_seed(args.seed, rank), T, V, w.id_dist)
-    st.ids = torch.from_numpy(ids_np).to(dev)
-    st.allocate(backward)
-    stream = torch.cuda.current_stream()
-    flops_step = layer_flops(T, d, F, backward)
-    run_step = lambda: st.step(backward=backward)
-    if args.variant == "dagger":
-        # STEM-dagger (Appendix): the up-projection is kept; 3 contractions forward, 6 backward
-        W_up = (torch.randn(F, d, generator=gen, device=dev, dtype=torch.float32) * d ** -0.5).to(dt)
-        U = torch.empty(T, F, dtype=dt, device=dev)
-        dW_up = torch.empty(F, d, dtype=torch.float32, device=dev)
-        flops_step = (18.0 if backward else 6.0) * T * d * F
-        b_ = st.bufs
-
-        def run_step():
-            st.dedup()
-            B.stem_dagger_forward(st.shape, st.x, st.ids, st.W_gate, W_up, st.E, st.W_down, b_["y"], b_["G"], b_["H"], U,
-                                  b_["ws"])
-            if backward:
-                B.stem_dagger_backward(st.shape, st.dy, st.x, st.W_gate, W_up, st.W_down, b_["G"], b_["H"], U, b_["perm"],
-                                       b_["seg_offsets"], b_["n_unique"], b_["dx"], b_["dW_gate"], dW_up, b_["dW_down"],
-                                       b_["dE_rows"], b_["ws"])
-
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing ------------------------------------------------------------
-    for _ in range(args.warmup):
-        run_step()
-    barrier()
-    assert st.status() == B.OK, B.status_string(st.status())
-    n_u = int(st.bufs["n_unique"].item())
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = B.stem_launch_count()
-    with ClockSampler(local) as clocks:
-        B.stem_profile_enable(not args.no_profile)
-        barrier()
-        t0 = time.time()
-        ev0.record(stream)
-        for _ in range(args.steps):
-            run_step()
-        ev1.record(stream)
-        barrier()
-        t1 = time.time()
-        B.stem_profile_enable(False)
-    launches = B.stem_launch_count() - launches0
-    ms_total = ev0.elapsed_time(ev1)
-    records = B.stem_profile_records()
-    assert st.status() == B.OK, B.status_string(st.status())
-    clock_summary = clocks.summary(t0, t1)
+    peaks = load_peaks()
+    T = args.tokens or w.T
+    head = measure_layer(w, T, args.steps, args.warmup, args, rank, local, dev, barrier, args.variant,
+                         profile=not args.no_profile)
+    st, n_u, ids_np = head["state"], head["n_unique"], head["ids_np"]
+    d, F, V, backward, dcode = w.d_model, w.d_ff, w.V, w.backward, head["dcode"]
+    esz = 2 if dcode == B.DTYPE_BF16 else 4
+    stream = torch.cuda.current_stream()
 
     # ---- end to end through the host-buffer entry point -------------------------------------
-    esz = 2 if dcode == B.DTYPE_BF16 else 4
     e2e = None
     if backward and not args.no_e2e and args.variant == "stem":
         hx, hdy = st.x.cpu().pin_memory(), st.dy.cpu().pin_memory()
@@ -814,28 +1064,32 @@ def main():
         assert int(hn[0]) == n_u
         assert torch.equal(hy, st.bufs["y"].cpu())       # same result as the device-resident path
         e2e = {"ms": e2e_ms, "h2d": 2 * T * d * esz + T * 4, "d2h": 2 * T * d * esz + 4}
-        del arena
+        # what the host link gives with both directions busy: plain pinned copies of the same sizes
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        dx_dev, dx2_dev = torch.empty_like(st.x), torch.empty_like(st.x)
+        torch.cuda.synchronize()
+        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0.record(stream)
+        s_in.wait_stream(stream); s_out.wait_stream(stream)
+        reps = 4
+        for _ in range(reps):
+            with torch.cuda.stream(s_in):
+                dx_dev.copy_(hx, non_blocking=True); dx2_dev.copy_(hdy, non_blocking=True)
+            with torch.cuda.stream(s_out):
+                hy.copy_(dx_dev, non_blocking=True); hdx.copy_(dx2_dev, non_blocking=True)
+        stream.wait_stream(s_in); stream.wait_stream(s_out)
+        l1.record(stream)
+        torch.cuda.synchronize()
+        e2e["link_ms"] = l0.elapsed_time(l1) / reps       # per step's worth of copies, both directions at once
+        del arena, dx_dev, dx2_dev
 
     # ---- compact row gather from the device-resident table (the standalone gather figure) ------------
     gather = None
     if rank == 0 and dcode == B.DTYPE_BF16:
-        cache = torch.empty(min(T, V), F, dtype=dt, device=dev)
-        b = st.bufs
-        for _ in range(3):
-            B.stem_prefetch_rows(st.shape, b["unique_ids"], b["n_unique"], st.E, cache, b["ws"])
-        torch.cuda.synchronize()
-        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = 20
-        g0.record(stream)
-        for _ in range(reps):
-            B.stem_prefetch_rows(st.shape, b["unique_ids"], b["n_unique"], st.E, cache, b["ws"])
-        g1.record(stream)
-        torch.cuda.synchronize()
-        g_ms = g0.elapsed_time(g1) / reps
-        gather = {"rows": n_u, "ms": g_ms, "bytes": 2 * n_u * F * esz}       # rows read once, written once
-        del cache
+        gather = measure_gather(st, n_u, T, V, F, esz, dev)
 
     # ---- max over ranks ------------------------------------------------------------------------
+    ms_total, launches = head["ms_total"], int(head["launches"])
     if world > 1:
         t = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0], dev)
         ms_total = t[0]
@@ -846,50 +1100,17 @@ def main():
             dist.destroy_process_group()
         return
 
-    peaks = load_peaks()
     ms_per_step = ms_total / args.steps
     value = world * T * args.steps / (ms_total * 1e-3)
-
-    # ---- per-kernel figures ------------------------------------------------------------------------
-    by_name: dict[str, list] = {}
-    for name, ms in records:
-        by_name.setdefault(name, []).append(ms)
-    flops_gemm = 2.0 * T * d * F
-    gbytes = 4 if st.shape.grad_dtype == B.DTYPE_FP32 else 2
-    seg_bytes = T * F * esz + n_u * F * gbytes + 4 * (T + n_u + 1)
-    kernels = {}
-    for name, v in by_name.items():
-        avg = float(np.mean(v))
-        k = {"launch_sets": len(v), "avg_ms": avg, "share": float(np.sum(v)) / ms_total}
-        if name.endswith("_gemm"):
-            k["tflops"] = flops_gemm / (avg * 1e-3) / 1e12
-            k["frac_of_measured_sustained"] = k["tflops"] / peaks["bf16_tflops_sustained"]
-            k["frac_of_measured_burst"] = k["tflops"] / peaks["bf16_tflops"]
-        elif name == "seg_reduce":
-            k["gbs"] = seg_bytes / (avg * 1e-3) / 1e9
-            k["frac_of_measured_hbm"] = k["gbs"] / peaks["hbm_gbs"]
-        kernels[name] = k
+    clock_summary = head["clocks"]
+    regime = roofline_regime(ms_total * 1e-3, clock_summary.get("sm_mhz"), peaks)
+    kernels = kernel_table(head["records"], ms_total, T, d, F, n_u, esz, st.shape.grad_dtype == B.DTYPE_FP32, peaks)
     if gather:
-        gbs = gather["bytes"] / (gather["ms"] * 1e-3) / 1e9
-        kernels["compact_gather"] = {"launch_sets": 20, "avg_ms": gather["ms"], "rows": gather["rows"], "gbs": gbs,
-                                     "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
-                                     "note": "cache[r] = E[unique_ids[r]] on the device, back to back, outside the timed step"}
+        kernels["compact_gather"] = gather_entry(gather, peaks)
     if "gate_gemm" in kernels:
         # rows the fused lookup hands to the epilogue, per second (not a roofline: the kernel is MMA-bound)
         kernels["gate_gemm"]["fused_lookup_gbs"] = T * F * esz / (kernels["gate_gemm"]["avg_ms"] * 1e-3) / 1e9
-    gemms = {n: k for n, k in kernels.items() if n.endswith("_gemm")}
-    roofline = None
-    if gemms and dcode == B.DTYPE_BF16:
-        dom = max(gemms, key=lambda n: gemms[n]["avg_ms"])
-        cap = load_traffic(dom)
-        # DRAM traffic grows in proportion to the tokens of a launch (every [T,.] operand does; the
-        # weights are the small remainder), so a capture at fewer tokens is scaled by T / T_captured.
-        traffic = cap[1] * T / cap[0] if cap else None
-        roofline = {"kernel": dom, "bound": "tensor", "achieved": gemms[dom]["tflops"],
-                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                    "frac": gemms[dom]["tflops"] / peaks["bf16_tflops_sustained"],
-                    "traffic": traffic, "peak_source": peaks["source"] + " (sustained bf16 GEMM, of measured)",
-                    "flops_per_launch": flops_gemm}
+    roofline, roofline_hbm = rooflines(kernels, regime, peaks, T, d, F, dcode == B.DTYPE_BF16)
 
     # ---- the CPU checker timed beside it (rank 0, N = 1 only) -----------------------------------------
     cpu = None
@@ -900,7 +1121,34 @@ def main():
                        "W_down": st.W_down.float().cpu().numpy(), "E": st.E.float().cpu().numpy()}
         tps, secs = oracle_tokens_per_sec(host_inputs, Tc)
         cpu = {"value": tps, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle", "seconds": secs,
+               "cores_note": "threads of the BLAS library numpy's matrix products run on",
                "sample": f"first {Tc} of {T} tokens, full weights and table, dedup + forward + backward in fp64"}
+
+    # ---- the other single-layer configurations, shorter, outside the headline's timed region --------
+    configs = None
+    if (world == 1 and args.workload == "1b" and args.variant == "stem" and not args.tokens and not args.no_configs):
+        configs = {}
+        del st, head
+        torch.cuda.empty_cache()
+        for name in ("350m", "1b_long_fwd"):
+            wc = synth.WORKLOADS[name]
+            steps_c = max(20, min(args.steps, 50))
+            m = measure_layer(wc, wc.T, steps_c, 5, args, rank, local, dev, barrier, "stem", profile=True)
+            es = 2
+            kern = kernel_table(m["records"], m["ms_total"], wc.T, wc.d_model, wc.d_ff, m["n_unique"], es, True, peaks)
+            g = measure_gather(m["state"], m["n_unique"], wc.T, wc.V, wc.d_ff, es, dev)
+            kern["compact_gather"] = gather_entry(g, peaks)
+            reg = roofline_regime(m["ms_total"] * 1e-3, m["clocks"].get("sm_mhz"), peaks)
+            rf, rf_hbm = rooflines(kern, reg, peaks, wc.T, wc.d_model, wc.d_ff, True)
+            ms_c = m["ms_total"] / steps_c
+            configs[name] = {
+                "T": wc.T, "d_model": wc.d_model, "d_ff": wc.d_ff, "V": wc.V, "ids": wc.id_dist, "backward": wc.backward,
+                "n_unique": m["n_unique"], "steps": steps_c, "warmup": 5, "ms_per_step": ms_c,
+                "value": wc.T / (ms_c * 1e-3), "unit": "tokens/s",
+                "tflops_step": layer_flops(wc.T, wc.d_model, wc.d_ff, wc.backward) / (ms_c * 1e-3) / 1e12,
+                "gpu_launches": m["launches"], "clocks": m["clocks"], "roofline": rf, "roofline_hbm": rf_hbm, "kernels": kern}
+            del m
+            torch.cuda.empty_cache()
 
     out = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -909,20 +1157,28 @@ def main():
         "config": {"workload": w.name, "T": T, "d_model": d, "d_ff": F, "V": V, "ids": w.id_dist,
                    "n_unique": n_u, "backward": backward, "variant": args.variant, "parallelism": f"replicas x{world}",
                    "l2": "per-step working set (~2.5 GB at 1b shapes) exceeds the 126 MB L2; no flush"},
-        "gpu_launches": int(launches),
-        "tflops_step": flops_step / (ms_per_step * 1e-3) / 1e12,
+        "gpu_launches": launches,
+        "tflops_step": layer_flops(T, d, F, backward) * (1.5 if args.variant == "dagger" else 1.0) / (ms_per_step * 1e-3) / 1e12,
         # the ids are the same for every STEM layer of a model, so their dedup can be paid once per batch
         "value_dedup_amortised": (world * T / ((ms_per_step - kernels["dedup"]["avg_ms"]) * 1e-3)
                                   if kernels.get("dedup") else None),
         "clocks": clock_summary,
         "roofline": roofline,
+        "roofline_hbm": roofline_hbm,
         "kernels": kernels,
         "cpu_baseline": cpu,
     }
+    if configs is not None:
+        out["configs"] = configs
     if e2e:
+        e2e_step = e2e["ms"] / args.steps
+        link_gbs = (e2e["h2d"] + e2e["d2h"]) / (e2e["link_ms"] * 1e-3) / 1e9
         out["e2e"] = {"value": world * T * args.steps / (e2e["ms"] * 1e-3), "unit": "tokens/s",
                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                      "ms_per_step": e2e["ms"] / args.steps}
+                      "ms_per_step": e2e_step,
+                      # the copies of a step, alone, both directions at once, against the kernels of a step
+                      "link_ms_per_step": e2e["link_ms"], "link_gbs_both_directions": link_gbs,
+                      "bound": "host link" if e2e["link_ms"] >= 0.9 * ms_per_step else "kernels"}
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

@@ -58,3 +58,32 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(r0.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0
+
+
+def test_roofline_regime_and_fractions():
+    """Host logic of the bench line: which measured peak a run is compared with, and that both
+    fractions, the nominal one and the HBM-bound kernels' figures are all carried."""
+    sys.path.insert(0, ROOT)
+    import bench
+    peaks = {"hbm_gbs": 6500.0, "bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0, "source": "measured",
+             "sm_mhz_under_load": 1340.0}
+    assert bench.roofline_regime(0.05, 1950.0, peaks) == "burst"          # too short to settle under the power cap
+    assert bench.roofline_regime(3.0, 1300.0, peaks) == "sustained"
+    assert bench.roofline_regime(3.0, 1900.0, peaks) == "burst"           # long, but at clocks far above the sustained run's
+    assert bench.roofline_regime(3.0, None, peaks) == "sustained"
+    T, d, F, n_u = 1000, 64, 128, 300
+    flops = 2.0 * T * d * F
+    # a contraction that takes exactly the time 800 TFLOP/s gives, a reduce at exactly 3250 GB/s
+    seg_bytes = T * F * 2 + n_u * F * 4 + 4 * (T + n_u + 1)
+    records = [("dh_gemm", flops / 800e12 * 1e3), ("down_gemm", flops / 1600e12 * 1e3), ("seg_reduce", seg_bytes / 3250e9 * 1e3)]
+    kern = bench.kernel_table(records, 1.0, T, d, F, n_u, 2, True, peaks)
+    assert abs(kern["dh_gemm"]["frac_of_measured_burst"] - 0.5) < 1e-9
+    assert abs(kern["dh_gemm"]["frac_of_nominal"] - 800.0 / 2250.0) < 1e-9
+    assert abs(kern["seg_reduce"]["frac_of_measured_hbm"] - 0.5) < 1e-9
+    rf, rf_hbm = bench.rooflines(kern, "burst", peaks, T, d, F, True)
+    assert rf["kernel"] == "dh_gemm" and rf["regime"] == "burst" and abs(rf["frac"] - 0.5) < 1e-9
+    assert abs(rf["frac_sustained"] - 800.0 / 1400.0) < 1e-9 and rf["peak"] == 1600.0
+    rf2, _ = bench.rooflines(kern, "sustained", peaks, T, d, F, True)
+    assert rf2["peak"] == 1400.0 and abs(rf2["frac"] - 800.0 / 1400.0) < 1e-9
+    assert rf_hbm["kernel"] == "seg_reduce" and rf_hbm["bound"] == "hbm" and abs(rf_hbm["frac"] - 0.5) < 1e-9
+    assert rf_hbm["bytes_per_launch"] == seg_bytes
