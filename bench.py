@@ -830,6 +830,14 @@ def shard_plan(V: int, world: int, rank: int) -> dict:
             "first_id": rank, "id_stride": world}
 
 
+def shard_rows_of_block(r0: int, r1: int, rank: int, world: int):
+    """Of the table rows [r0, r1) drawn as one block, which belong to `rank` (id mod world == rank):
+    (offset of the first one inside the block, its local row index, how many)."""
+    first = (rank - r0) % world
+    count = len(range(r0 + first, r1, world))
+    return first, (r0 + first) // world, count
+
+
 def sharded_line(args, w, T, world, ms_total, phase_ms, plan, sent, launches, clocks) -> dict:
     """The JSON line of the sharded mode from rank 0's view: times are maxima over ranks already."""
     F = w.d_ff
@@ -891,10 +899,8 @@ def run_sharded_dist(args, w):
     for r0 in range(0, V, 4096):                                     # the whole table is drawn, this rank keeps its rows
         r1 = min(V, r0 + 4096)
         blk = (torch.randn(r1 - r0, F, generator=gen, device=dev) * 0.02).to(dt)
-        first = (rank - r0) % world                                   # first row of the block with id mod world == rank
-        mine = blk[first::world]
-        lo = (r0 + first) // world
-        shard[lo:lo + mine.shape[0]] = mine
+        first, lo, count = shard_rows_of_block(r0, r1, rank, world)
+        shard[lo:lo + count] = blk[first::world]
     gen_r = torch.Generator(device=dev).manual_seed(args.seed + 1000 * (rank + 1))    # the batch: every rank its own
     x = torch.randn(T, d, generator=gen_r, device=dev).to(dt)
     dy = torch.randn(T, d, generator=gen_r, device=dev).to(dt)

@@ -22,7 +22,7 @@ constexpr int kSegBlk = 64;     // most sorted positions per CTA (the launch pic
 constexpr int kCtasPerSm = 7;   // register budget the kernel is compiled for
 constexpr int kThreads = 128;   // pass 1: one thread per vector of columns
 constexpr int kBatch = 8;       // rows requested before the first is consumed
-constexpr int kFinBatch = 8;    // finishing kernel: partial rows requested before the first is added
+constexpr int kFinBatch = 16;    // finishing kernel: partial rows requested before the first is added
 
 template <typename T> struct Vec;
 template <> struct Vec<float> {
@@ -127,22 +127,28 @@ segreduce_kernel(int T, int F, int blk_len, const TIn* __restrict__ dU, const in
 #pragma unroll
   for (int i = 0; i < VI; ++i) acc[i] = 0.0f;
   bool first_run = true;
-  for (int b0 = 0; col_ok && b0 < cnt; b0 += kBatch) {
-    uint4 raw[kBatch][LD];
+  // Rows are requested kHalf at a time, two requests in flight: while one half-batch is being
+  // added, the next one is already on its way, so a thread never sits without loads outstanding
+  // (the memory system, not the adds, sets the pace of this kernel).
+  constexpr int kHalf = kBatch / 2;
+  uint4 raw[2][kHalf][LD];
+  auto request = [&](int buf, int first) {
 #pragma unroll
-    for (int j = 0; j < kBatch; ++j) {
-      if (b0 + j < cnt) {
-        const TIn* src = dU + static_cast<size_t>(s_row[b0 + j]) * F + col;
+    for (int j = 0; j < kHalf; ++j) {
+      if (first + j < cnt) {
+        const TIn* src = dU + static_cast<size_t>(s_row[first + j]) * F + col;
 #pragma unroll
-        for (int i = 0; i < LD; ++i) raw[j][i] = Vec<TIn>::load_raw(src + i * Vec<TIn>::N);
+        for (int i = 0; i < LD; ++i) raw[buf][j][i] = Vec<TIn>::load_raw(src + i * Vec<TIn>::N);
       }
     }
+  };
+  auto consume = [&](int buf, int first) {
 #pragma unroll
-    for (int j = 0; j < kBatch; ++j) {
-      const int q = b0 + j;
+    for (int j = 0; j < kHalf; ++j) {
+      const int q = first + j;
       if (q < cnt) {
 #pragma unroll
-        for (int i = 0; i < LD; ++i) Vec<TIn>::add(acc + i * Vec<TIn>::N, raw[j][i]);
+        for (int i = 0; i < LD; ++i) Vec<TIn>::add(acc + i * Vec<TIn>::N, raw[buf][j][i]);
         const int loc = s_loc[q];
         const bool run_ends = (q + 1 == cnt) || (s_loc[q + 1] != loc);
         if (run_ends) {
@@ -158,6 +164,15 @@ segreduce_kernel(int T, int F, int blk_len, const TIn* __restrict__ dU, const in
         }
       }
     }
+  };
+  if (col_ok) {
+    request(0, 0);
+    for (int b0 = 0; b0 < cnt; b0 += kBatch) {
+      request(1, b0 + kHalf);
+      consume(0, b0);
+      request(0, b0 + kBatch);
+      consume(1, b0 + kHalf);
+    }
   }
 
   // ---- the note for the finishing kernel: the crossing segment that starts in this block ------
@@ -169,11 +184,12 @@ segreduce_kernel(int T, int F, int blk_len, const TIn* __restrict__ dU, const in
   }
 }
 
-// Finishing kernel: one CTA per (block, column slab).  If a crossing segment starts in the block,
-// add its partial rows in block order and write the row.
+// Finishing kernel: one CTA per (block, slab of 4 * kThreads columns), one 4-column vector per
+// thread.  If a crossing segment starts in the block, add its partial rows in block order and
+// write the row.
 template <typename TOut>
 __global__ void __launch_bounds__(kThreads)
-segfinish_kernel(int F, int blk_len, int vi, const int4* __restrict__ notes, const float* __restrict__ partial,
+segfinish_kernel(int F, int blk_len, const int4* __restrict__ notes, const float* __restrict__ partial,
                  TOut* __restrict__ dE_rows) {
   ptx::grid_dependency_wait();
   ptx::grid_launch_dependents();
@@ -181,35 +197,31 @@ segfinish_kernel(int F, int blk_len, int vi, const int4* __restrict__ notes, con
   if (note.x < 0) return;
   const int seg_begin = note.y, seg_end = note.z;
   const int start_blk = blockIdx.x, last_blk = (seg_end - 1) / blk_len;
-  // the same columns per thread as in the first kernel: vi consecutive columns, in groups of 4
-  const int col0 = (blockIdx.y * kThreads + threadIdx.x) * vi;
-  if (col0 >= F) return;
-  for (int c = 0; c < vi; c += 4) {
-    const int col = col0 + c;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    // parts are requested kFinBatch at a time and added in block order: a segment of a frequent id
-    // spans dozens of blocks, and one load latency per block would make this launch a serial tail
-    for (int b0 = start_blk; b0 <= last_blk; b0 += kFinBatch) {
-      float4 q[kFinBatch];
+  const int col = (blockIdx.y * kThreads + threadIdx.x) * 4;
+  if (col >= F) return;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  // parts are requested kFinBatch at a time and added in block order: a segment of a frequent id
+  // spans dozens of blocks, and one load latency per block would make this launch a serial tail
+  for (int b0 = start_blk; b0 <= last_blk; b0 += kFinBatch) {
+    float4 q[kFinBatch];
 #pragma unroll
-      for (int i = 0; i < kFinBatch; ++i) {
-        const int b = b0 + i;
-        if (b <= last_blk) {
-          // the segment's run is the first run of block b, unless b is the block it starts in
-          // and it does not start at that block's first position
-          const int slot = (b > start_blk || seg_begin == start_blk * blk_len) ? 2 * b : 2 * b + 1;
-          q[i] = __ldcg(reinterpret_cast<const float4*>(partial + static_cast<size_t>(slot) * F + col));
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < kFinBatch; ++i) {
-        if (b0 + i <= last_blk) { acc.x += q[i].x; acc.y += q[i].y; acc.z += q[i].z; acc.w += q[i].w; }
+    for (int i = 0; i < kFinBatch; ++i) {
+      const int b = b0 + i;
+      if (b <= last_blk) {
+        // the segment's run is the first run of block b, unless b is the block it starts in
+        // and it does not start at that block's first position
+        const int slot = (b > start_blk || seg_begin == start_blk * blk_len) ? 2 * b : 2 * b + 1;
+        q[i] = __ldcg(reinterpret_cast<const float4*>(partial + static_cast<size_t>(slot) * F + col));
       }
     }
-    TOut* dst = dE_rows + static_cast<size_t>(note.x) * F + col;
-    dst[0] = from_f32<TOut>(acc.x); dst[1] = from_f32<TOut>(acc.y);
-    dst[2] = from_f32<TOut>(acc.z); dst[3] = from_f32<TOut>(acc.w);
+#pragma unroll
+    for (int i = 0; i < kFinBatch; ++i) {
+      if (b0 + i <= last_blk) { acc.x += q[i].x; acc.y += q[i].y; acc.z += q[i].z; acc.w += q[i].w; }
+    }
   }
+  TOut* dst = dE_rows + static_cast<size_t>(note.x) * F + col;
+  dst[0] = from_f32<TOut>(acc.x); dst[1] = from_f32<TOut>(acc.y);
+  dst[2] = from_f32<TOut>(acc.z); dst[3] = from_f32<TOut>(acc.w);
 }
 
 // Resident CTAs of the first kernel per SM, per device (an occupancy query is not free).
@@ -258,7 +270,8 @@ cudaError_t launch_typed(int T, int F, const void* dU, const int32_t* perm, cons
                                      seg_offsets, n_unique, static_cast<TOut*>(dE_rows), notes, partial);
   count_launches(1);
   if (e != cudaSuccess) return e;
-  e = cudaLaunchKernelEx(&cfg, segfinish_kernel<TOut>, F, blk_len, VI, static_cast<const int4*>(notes),
+  cfg.gridDim = dim3(n_blk, (F + 4 * kThreads - 1) / (4 * kThreads));
+  e = cudaLaunchKernelEx(&cfg, segfinish_kernel<TOut>, F, blk_len, static_cast<const int4*>(notes),
                          static_cast<const float*>(partial), static_cast<TOut*>(dE_rows));
   count_launches(1);
   return e != cudaSuccess ? e : cudaGetLastError();

@@ -87,3 +87,47 @@ def test_roofline_regime_and_fractions():
     assert rf2["peak"] == 1400.0 and abs(rf2["frac"] - 800.0 / 1400.0) < 1e-9
     assert rf_hbm["kernel"] == "seg_reduce" and rf_hbm["bound"] == "hbm" and abs(rf_hbm["frac"] - 0.5) < 1e-9
     assert rf_hbm["bytes_per_launch"] == seg_bytes
+
+
+def _sharded_plumbing_rank(rank: int, world: int, port: int, out_dir: str):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    sys.path.insert(0, ROOT)
+    import argparse
+    import bench
+    from paper_2601_10639_b200 import synth
+    V = 1003
+    plan = bench.shard_plan(V, world, rank)
+    # the table is drawn block by block; a rank keeps its rows of each block: together they must be E[rank::world]
+    table = torch.arange(V * 2, dtype=torch.float32).reshape(V, 2)
+    shard = torch.full((plan["rows_owned"], 2), -1.0)
+    for r0 in range(0, V, 100):
+        r1 = min(V, r0 + 100)
+        first, lo, count = bench.shard_rows_of_block(r0, r1, rank, world)
+        shard[lo:lo + count] = table[r0:r1][first::world]
+    ok = bool(torch.equal(shard, table[rank::world]))
+    # times are maxima over ranks; only rank 0 assembles (and prints) the line
+    t = bench.max_over_ranks([4.0 + rank, 1.0, 2.0 - rank], torch.device("cpu"))
+    line = None
+    if rank == 0:
+        args = argparse.Namespace(steps=2, warmup=3)
+        w = synth.WORKLOADS["350m"]
+        line = bench.sharded_line(args, w, 64, world, t[0], {"route": t[1], "layer": t[2]}, plan, [5, 7], 40,
+                                  {"sm_mhz": None})
+    with open(os.path.join(out_dir, f"s{rank}.json"), "w") as f:
+        json.dump({"ok": ok, "rows": plan["rows_owned"], "line": line}, f)
+    dist.destroy_process_group()
+
+
+def test_sharded_mode_rank_plumbing_two_gloo_ranks(tmp_path):
+    mp.spawn(_sharded_plumbing_rank, args=(2, _free_port(), str(tmp_path)), nprocs=2, join=True)
+    got = [json.load(open(tmp_path / f"s{r}.json")) for r in range(2)]
+    assert got[0]["ok"] and got[1]["ok"]
+    assert got[0]["rows"] + got[1]["rows"] == 1003 and got[0]["rows"] == 502
+    assert got[1]["line"] is None
+    line = got[0]["line"]
+    assert line["n_gpus"] == 2 and line["config"]["parallelism"].startswith("table sharded id mod 2")
+    assert line["ms_per_step"] == 5.0 / 2 and line["value"] == 2 * 64 * 2 / 5.0e-3       # slowest rank's time, all ranks' tokens
+    assert line["rank0_rows"] == {"distinct": 12, "from_other_ranks": 7}
+    assert line["rank0_exchange_bytes"]["rows_in"] == 7 * 2816 * 2
+    assert line["ms_per_phase_max_over_ranks"] == {"route": 1.0, "layer": 2.0}
