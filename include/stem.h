@@ -17,7 +17,11 @@
  *     The caller owns every buffer, the workspace included.  The library allocates no
  *     device memory.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
- *     only enqueue work; they do not synchronise unless stated.
+ *     only enqueue work; they do not synchronise unless stated.  Calls are re-entrant across
+ *     distinct workspaces.  On ONE workspace, issue them on one stream in the documented order:
+ *     the regions of a workspace are shared between calls (stem_dedup_ids' sort scratch, the H
+ *     of a forward call that was given no H_save, and backward's dU / dG all start at the same
+ *     offset), so e.g. stem_dedup_ids on a workspace destroys an unsaved H that still lives in it.
  *   - Outputs are overwritten, except the weight gradients under STEM_FLAG_ACCUM_GRADS.
  *   - Return value: STEM_OK or a negative STEM_ERR_* code.  Conditions only the device
  *     can see (an id outside [0,V), a pipeline wait that ran out) are recorded in the
@@ -63,6 +67,13 @@ extern "C" {
  * rows of dE_rows belong to this call's unique ids).  With bf16 gradients the product is rounded
  * to bf16 before the bf16 add. */
 #define STEM_FLAG_ACCUM_GRADS 4
+/* stem_dagger_forward: compute the gate and up products of x in ONE launch with two accumulators in
+ * tensor memory (U = up + E[ids] and H = SiLU(gate) (.) U formed in its epilogue) instead of two
+ * launches that pass U through memory.  Same results within rounding (H is formed from the
+ * unrounded U).  Saves one pass over x and one read of U; measured slower on B200 at the 1B shape
+ * (the tile must shrink to 256 x 128 per product and shared-memory bandwidth binds), so it is off by
+ * default.  CTA pairs only: ignored with STEM_FLAG_SINGLE_CTA or STEM_FLAG_SIMT. */
+#define STEM_FLAG_DAGGER_FUSED 8
 
 typedef struct {
   int32_t T;          /* positions in this call (batch x sequence)                 */
@@ -175,7 +186,7 @@ int stem_ffn_backward(const stem_shape_t* shape, const void* dy, const void* x, 
  * up-projection and adds the token's table row to its output):
  *     y_t = W_down ( SiLU(W_gate x_t) (.) (W_up x_t + E[id_t]) )
  * Forward: U = x W_up^T + E[ids] (the lookup is added in the up GEMM's epilogue), G = x W_gate^T,
- * H = SiLU(G) (.) U, y = H W_down^T.  W_up [d_ff,d_model] like W_gate.  U_save [T,d_ff] (dtype) is
+ * H = SiLU(G) (.) U, y = H W_down^T (STEM_FLAG_DAGGER_FUSED: the first three in one launch).  W_up [d_ff,d_model] like W_gate.  U_save [T,d_ff] (dtype) is
  * a required output (the backward pass needs it); G_save, H_save as in stem_ffn_forward.
  * Backward (chain rule, as for the layer itself): dH = dy W_down; dU = dH (.) SiLU(G);
  * dG = dH (.) U (.) SiLU'(G); dW_down = dy^T H; dW_gate = dG^T x; dW_up = dU^T x;

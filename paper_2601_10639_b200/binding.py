@@ -26,6 +26,7 @@ DTYPE_FP32, DTYPE_BF16 = 0, 1
 FLAG_SIMT = 1
 FLAG_SINGLE_CTA = 2
 FLAG_ACCUM_GRADS = 4
+FLAG_DAGGER_FUSED = 8
 
 EXPORTS = (
     "stem_version", "stem_status_string", "stem_workspace_bytes", "stem_init_workspace",

@@ -412,20 +412,34 @@ int stem_dagger_forward(const stem_shape_t* shape, const void* x, const int32_t*
   const int T = shape->T, d = shape->d_model, F = shape->d_ff;
   void* H = H_save ? H_save : static_cast<char*>(ws) + w.h_off;
   cudaError_t e;
-  {  // U = x W_up^T + E[ids]: the lookup is added in the up GEMM's epilogue
-    EpiParams up;
-    up.ids = ids; up.E = E; up.V = shape->V; up.H = U_save; up.status = status_of(ws);
-    ProfScope prof("up_gemm", st);
-    e = gemm(shape, T, F, d, x, false, W_up, false, kEpiAdd, up, st);
+  if (use_tc(shape) && (shape->flags & STEM_FLAG_DAGGER_FUSED) && !(shape->flags & STEM_FLAG_SINGLE_CTA)) {
+    // One kernel for both products of x: the gate and up tiles of the same x rows accumulate side
+    // by side in tensor memory, and the epilogue forms U = up + E[ids], H = SiLU(gate) (.) U in
+    // registers.  x is streamed once, and U reaches memory only as the copy backward needs.
+    // Opt-in: two accumulator sets leave room for 128-column tiles only, every A block is then read
+    // from shared memory once per product, and shared-memory bandwidth makes this launch about a
+    // fifth slower than the two launches it replaces (measured at the 1B shape).
+    EpiParams du;
+    du.ids = ids; du.E = E; du.V = shape->V; du.H = H; du.G = G_save; du.U = U_save; du.status = status_of(ws);
+    ProfScope prof("gate_up_gemm", st);
+    e = launch_tc_gemm_dagger(T, F, d, x, W_gate, W_up, du, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  } else {
+    {  // U = x W_up^T + E[ids]: the lookup is added in the up GEMM's epilogue
+      EpiParams up;
+      up.ids = ids; up.E = E; up.V = shape->V; up.H = U_save; up.status = status_of(ws);
+      ProfScope prof("up_gemm", st);
+      e = gemm(shape, T, F, d, x, false, W_up, false, kEpiAdd, up, st);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    {  // G = x W_gate^T, H = SiLU(G) (.) U: the gate epilogue with U as a [T, d_ff] "table" indexed by position
+      EpiParams gate;
+      gate.ids = nullptr; gate.E = U_save; gate.V = T; gate.H = H; gate.G = G_save; gate.status = status_of(ws);
+      ProfScope prof("gate_gemm", st);
+      e = gemm(shape, T, F, d, x, false, W_gate, false, kEpiGate, gate, st);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
   }
-  if (e != cudaSuccess) return cuda_fail(e);
-  {  // G = x W_gate^T, H = SiLU(G) (.) U: the gate epilogue with U as a [T, d_ff] "table" indexed by position
-    EpiParams gate;
-    gate.ids = nullptr; gate.E = U_save; gate.V = T; gate.H = H; gate.G = G_save; gate.status = status_of(ws);
-    ProfScope prof("gate_gemm", st);
-    e = gemm(shape, T, F, d, x, false, W_gate, false, kEpiGate, gate, st);
-  }
-  if (e != cudaSuccess) return cuda_fail(e);
   EpiParams down;
   down.out = y; down.out_fp32 = shape->dtype == STEM_DTYPE_FP32; down.status = status_of(ws);
   down.sk_scratch = static_cast<char*>(ws) + w.sk_off; down.sk_bytes = w.sk_bytes;

@@ -44,14 +44,16 @@ constexpr int kAtomBytes = 64 * BK * 2;                // one 64(MN) x BK swizzl
 // CTAS = 2: two CTAs of a cluster share every MMA (cta_group::2).  Each stages its own 128
 // rows of A and half of the BN columns of B, so a stage is 32 KB instead of 48 KB and the
 // operand bytes fetched per flop drop by a third.
-template <int BN, int STAGES, int CTAS>
+// DUAL: two products of the same A tile per stage (B operands of both, side by side) and three
+// output blocks per epilogue warp.
+template <int BN, int STAGES, int CTAS, bool DUAL = false>
 struct Smem {
   static constexpr int kABytes = BM * BK * 2;
-  static constexpr int kBBytes = (BN / CTAS) * BK * 2;
-  static constexpr int kStageBytes = kABytes + kBBytes;
-  // per epilogue warp: two 2 KB output blocks (32 rows x 32 bf16) or one 4 KB block (fp32)
+  static constexpr int kBBytes = (BN / CTAS) * BK * 2;          // one B operand
+  static constexpr int kStageBytes = kABytes + (DUAL ? 2 : 1) * kBBytes;
+  // per epilogue warp: two (DUAL: three) 2 KB output blocks (32 rows x 32 bf16) or one 4 KB block (fp32)
   static constexpr int kOutOffset = STAGES * kStageBytes;
-  static constexpr int kOutBytesPerWarp = 4096;
+  static constexpr int kOutBytesPerWarp = DUAL ? 6144 : 4096;
   static constexpr int kBarOffset = kOutOffset + kEpiWarps * kOutBytesPerWarp;
   // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain, tmem address, abort
   static constexpr int kNumBars = 2 * STAGES + 5;
@@ -134,6 +136,25 @@ __device__ __forceinline__ void stage_row_f32(uint32_t buf, int lane, const uint
 // Fused elementwise step on 32 consecutive columns of one output row: results go to the
 // warp's staging buffer (first output at buf, second at buf + 2048).  e and g hold the
 // table row segment and the saved pre-activation (bf16 pairs), fetched earlier.
+// kEpiDagger: acc = the gate product, up = the up product of the same 32 columns:
+// U = up + E[id], H = SiLU(acc) * U; outputs H, then (optional) G = acc and U.
+__device__ __forceinline__ void epilogue_row32_dagger(const EpiParams& ep, uint32_t buf, int lane,
+                                                      const uint32_t (&acc)[32], const uint32_t (&up)[32],
+                                                      const uint32_t (&e)[16]) {
+  uint32_t h[16], go[16], uo[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float a0 = __uint_as_float(acc[2 * i]), a1 = __uint_as_float(acc[2 * i + 1]);
+    const float u0 = __uint_as_float(up[2 * i]) + bf16_lo(e[i]), u1 = __uint_as_float(up[2 * i + 1]) + bf16_hi(e[i]);
+    h[i] = pack_bf16(a0 * fast_sigmoid(a0) * u0, a1 * fast_sigmoid(a1) * u1);
+    go[i] = pack_bf16(a0, a1);
+    uo[i] = pack_bf16(u0, u1);
+  }
+  stage_row_bf16(buf, lane, h);
+  if (ep.G) stage_row_bf16(buf + 2048, lane, go);
+  if (ep.U) stage_row_bf16(buf + 4096, lane, uo);
+}
+
 template <int KIND>
 __device__ __forceinline__ void epilogue_row32(const EpiParams& ep, uint32_t buf, int lane,
                                                const uint32_t (&acc)[32], const uint32_t (&e)[16],
@@ -222,7 +243,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
                const __grid_constant__ CUtensorMap tmC2,
                int M, int N, int K, int M2, int N2, int group_m, int dp_tiles, int split, EpiParams ep) {
-  using L = Smem<BN, STAGES, CTAS>;
+  constexpr bool kDual = KIND == kEpiDagger;      // two products (gate, up) of every A tile
+  using L = Smem<BN, STAGES, CTAS, kDual>;
+  constexpr int kAccCols = kDual ? 2 * BN : BN;   // TMEM columns of one accumulator set
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -249,7 +272,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int num_tiles1 = tiles_m * tiles_n;
   const int num_tiles = num_tiles1 + tiles_m2 * tiles_n2;
   const int k_blocks = (K + BK - 1) / BK;
-  constexpr uint32_t kTmemCols = 2 * BN;
+  constexpr uint32_t kTmemCols = 2 * kAccCols;
+  static_assert(kTmemCols <= 512, "two accumulator sets must fit the 512 TMEM columns");
   const WorkList work{unit0, unit_stride, dp_tiles, num_tiles, k_blocks, split};
 
   if (threadIdx.x == 0) {
@@ -261,7 +285,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
     ptx::prefetch_tensormap(&tmC0);
-    if (KIND == kEpiGate || KIND == kEpiDH) ptx::prefetch_tensormap(&tmC1);
+    if (KIND == kEpiGate || KIND == kEpiDH || kDual) ptx::prefetch_tensormap(&tmC1);
+    if (kDual) { ptx::prefetch_tensormap(&tmB2); ptx::prefetch_tensormap(&tmC2); }
     if (KIND == kEpiStore && M2 > 0) {
       ptx::prefetch_tensormap(&tmA2);
       ptx::prefetch_tensormap(&tmB2);
@@ -327,6 +352,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int j = 0; j < BN / CTAS / 64; ++j) load(b_dst + j * kAtomBytes, mapB, n0 + 64 * j, k0);
           } else {
             load(b_dst, mapB, k0, n0);
+            if (kDual) load(b_dst + L::kBBytes, &tmB2, k0, n0);    // the up-projection's rows of the same columns
           }
           ++issued;
           if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -349,7 +375,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           *abort_flag = 1; ok = false; break;
         }
         ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * BN;
+        const uint32_t d_tmem = tmem_base + acc * kAccCols;
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, kWaitLimitCycles)) {
             report_error(ep.status, STEM_ERR_TIMEOUT, 2);
@@ -370,6 +396,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (CTAS == 2) ptx::mma_bf16_ss_pair(d_tmem, ad, bd, idesc, (kb > w.kb0 || kk > 0) ? 1u : 0u);
             else ptx::mma_bf16_ss(d_tmem, ad, bd, idesc, (kb > w.kb0 || kk > 0) ? 1u : 0u);
           }
+          if (kDual) {   // the same A block against the second B operand, into the second accumulator
+#pragma unroll
+            for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+              const uint64_t ad = ptx::make_smem_desc(a_src + kk * (UMMA_K * 2), 16, 1024);
+              const uint64_t bd2 = ptx::make_smem_desc(b_src + L::kBBytes + kk * (UMMA_K * 2), 16, 1024);
+              if (CTAS == 2) ptx::mma_bf16_ss_pair(d_tmem + BN, ad, bd2, idesc, (kb > w.kb0 || kk > 0) ? 1u : 0u);
+              else ptx::mma_bf16_ss(d_tmem + BN, ad, bd2, idesc, (kb > w.kb0 || kk > 0) ? 1u : 0u);
+            }
+          }
           commit(empty_bar(s));
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
@@ -389,7 +424,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int half = (warp - 2) >> 2;       // which half of the tile's columns it handles
     constexpr int kChunks = BN / 2 / 32;    // 32-column chunks per thread per tile
     const uint32_t out_buf = base + L::kOutOffset + (warp - 2) * L::kOutBytesPerWarp;
-    const bool second_out = KIND == kEpiDH || (KIND == kEpiGate && ep.G != nullptr);
+    const bool second_out = KIND == kEpiDH || ((KIND == kEpiGate || kDual) && ep.G != nullptr);
     constexpr bool kReadOnlyE = KIND != kEpiAdd;   // the add epilogue may overwrite its addend
     int acc = 0; uint32_t aph = 0;
     bool ok = true;
@@ -429,7 +464,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         ok = false; break;
       }
       ptx::tc_fence_after();
-      const uint32_t t_row = tmem_base + acc * BN + half * (BN / 2) + (static_cast<uint32_t>(q * 32) << 16);
+      const uint32_t t_row = tmem_base + acc * kAccCols + half * (BN / 2) + (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll
       for (int c = 0; c < kChunks; ++c) {
         uint32_t e_cur[16], g_cur[16];
@@ -440,8 +475,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           load_bf16x32<WIDE, kReadOnlyE>(e_row + n + 32, n + 32, N, e_next);
           if (KIND == kEpiDH) load_bf16x32<WIDE>(g_row + n + 32, n + 32, N, g_next);
         }
-        uint32_t v[32];
+        uint32_t v[32], v2[kDual ? 32 : 1];
         ptx::tmem_ld_32x32(t_row + c * 32, v);
+        if constexpr (kDual) ptx::tmem_ld_32x32(t_row + BN + c * 32, v2);
         ptx::tmem_ld_wait();
         if (c + 1 == kChunks) {
           // the accumulator has been read out: hand it back to the MMA issuer
@@ -465,13 +501,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ptx::bulk_commit_group();
           }
         } else {
-          epilogue_row32<KIND>(ep, out_buf, lane, v, e_cur, g_cur);
+          if constexpr (kDual) epilogue_row32_dagger(ep, out_buf, lane, v, v2, e_cur);
+          else epilogue_row32<KIND>(ep, out_buf, lane, v, e_cur, g_cur);
           ptx::fence_proxy_async();
           __syncwarp();
           if (lane == 0 && m_warp < M_ && n < N_) {
             if (KIND == kEpiStore && ep.accumulate) ptx::tma_reduce_add_2d(mapC, out_buf, n, m_warp);
             else ptx::tma_store_2d(mapC, out_buf, n, m_warp);
             if (second_out) ptx::tma_store_2d(&tmC1, out_buf + 2048, n, m_warp);
+            if (kDual && ep.U != nullptr) ptx::tma_store_2d(&tmC2, out_buf + 4096, n, m_warp);
             ptx::bulk_commit_group();
           }
         }
@@ -617,13 +655,15 @@ bool encode_out_map(CUtensorMap* map, const void* ptr, int rows, int cols, bool 
 
 // A second product C2 = A2 B2^T with the same contraction length and operand layouts, carried by
 // the same launch (plain stores only); M == 0 means none.
-struct SecondMaps { CUtensorMap A, B, C; int M = 0, N = 0; void* out = nullptr; };
+// The same parameter slots carry the second B operand (B) and the third output (C) of the
+// two-product kind kEpiDagger, with M == 0 and `maps` set.
+struct SecondMaps { CUtensorMap A, B, C; int M = 0, N = 0; void* out = nullptr; bool maps = false; };
 
 template <bool A_MN, bool B_MN, int KIND, int BN, int STAGES, bool WIDE, int CTAS>
 cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC0,
                         const CUtensorMap& tmC1, int M, int N, int K, const EpiParams& ep, int sk_tail,
                         int sk_split, const SecondMaps& sec, cudaStream_t stream) {
-  using L = Smem<BN, STAGES, CTAS>;
+  using L = Smem<BN, STAGES, CTAS, KIND == kEpiDagger>;
   static_assert(L::kTotal <= 232448, "exceeds the shared memory a CTA can have");
   auto kern = tc_gemm_kernel<A_MN, B_MN, KIND, BN, STAGES, WIDE, CTAS>;
   static PerDeviceOnce configured;
@@ -652,8 +692,9 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC0, tmC1, sec.M > 0 ? sec.A : tmA, sec.M > 0 ? sec.B : tmB,
-                                     sec.M > 0 ? sec.C : tmC0, M, N, K, sec.M, sec.N, 8, dp_tiles, sk_split, ep);
+  const bool second_maps = sec.M > 0 || sec.maps;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmC0, tmC1, sec.M > 0 ? sec.A : tmA, second_maps ? sec.B : tmB,
+                                     second_maps ? sec.C : tmC0, M, N, K, sec.M, sec.N, 8, dp_tiles, sk_split, ep);
   count_launches(1);
   if (e == cudaSuccess && sk_tail > 0) {
     cudaLaunchConfig_t fcfg = {};
@@ -738,6 +779,27 @@ cudaError_t launch_ctas(const void* A, const void* B, int M, int N, int K, const
 }
 
 }  // namespace
+
+cudaError_t launch_tc_gemm_dagger(int M, int N, int K, const void* A, const void* B_gate, const void* B_up,
+                                  const EpiParams& ep, cudaStream_t stream) {
+  if (M <= 0 || N <= 0) return cudaSuccess;
+  if (K <= 0 || (N % 8) || (K % 8)) return cudaErrorNotSupported;
+  // CTA pairs; 256 x 128 tiles of BOTH products: 2 x 2 x 128 accumulator columns fill TMEM, and a
+  // stage holds the A block and the two B blocks (32 KB per CTA), five stages deep
+  constexpr int BN = 128, STAGES = 5, CTAS = 2;
+  CUtensorMap tmA, tmB, tmC0, tmC1;
+  SecondMaps sec;
+  sec.maps = true;
+  bool ok = encode_map(&tmA, A, M, K, BM) && encode_map(&tmB, B_gate, N, K, BN / CTAS) &&
+            encode_map(&sec.B, B_up, N, K, BN / CTAS) && encode_out_map(&tmC0, ep.H, M, N, false);
+  if (ep.G) ok = ok && encode_out_map(&tmC1, ep.G, M, N, false); else tmC1 = tmC0;
+  if (ep.U) ok = ok && encode_out_map(&sec.C, ep.U, M, N, false); else sec.C = tmC0;
+  if (!ok) return cudaErrorNotSupported;
+  auto a32 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; };
+  if ((N % 16 == 0) && a32(ep.E))
+    return launch_inst<false, false, kEpiDagger, BN, STAGES, true, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, 0, 1, sec, stream);
+  return launch_inst<false, false, kEpiDagger, BN, STAGES, false, CTAS>(tmA, tmB, tmC0, tmC1, M, N, K, ep, 0, 1, sec, stream);
+}
 
 cudaError_t launch_tc_gemm_token_pair(int K, int M1, int N1, const void* A1, const void* B1, void* out1, int M2,
                                       int N2, const void* A2, const void* B2, void* out2, const EpiParams& ep,

@@ -36,7 +36,7 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
 __device__ __forceinline__ float sigmoid_f32(float g) { return 1.0f / (1.0f + expf(-g)); }
 
 // ---- epilogue descriptions (shared by the FMA and the tensor-core GEMM front ends) ---
-enum EpiKind : int { kEpiStore = 0, kEpiGate = 1, kEpiDH = 2, kEpiAdd = 3 };
+enum EpiKind : int { kEpiStore = 0, kEpiGate = 1, kEpiDH = 2, kEpiAdd = 3, kEpiDagger = 4 };
 
 struct EpiParams {
   // kEpiStore: out[m*ld + n] = acc              (out_fp32 selects fp32 or bf16/T storage)
@@ -55,6 +55,9 @@ struct EpiParams {
   void* H = nullptr;    // kEpiGate: H out          kEpiDH: dU out
   void* G = nullptr;    // kEpiGate: G out (opt.)   kEpiDH: dG out
   const void* Gin = nullptr;  // kEpiDH: saved G
+  // kEpiDagger (two products of the same A tile, gate = acc and up = acc2):
+  //            U = acc2 + E[ids[m], n]; H = SiLU(acc) * U; optional G = acc, optional U out
+  void* U = nullptr;
   int32_t* status = nullptr;
   // kEpiStore, optional: scratch for partial tiles when the last round of tiles is split
   // along k (tc_gemm_scratch_bytes()); without it every tile is computed whole
@@ -82,6 +85,12 @@ cudaError_t launch_tc_gemm(int M, int N, int K, const void* A, bool a_mn, const 
 cudaError_t launch_tc_gemm_token_pair(int K, int M1, int N1, const void* A1, const void* B1, void* out1, int M2,
                                       int N2, const void* A2, const void* B2, void* out2, const EpiParams& ep,
                                       bool pair, cudaStream_t stream);
+
+// The dagger variant's gate and up products of the same x tile in one launch (CTA pairs, two
+// accumulators): G = A B_gate^T, Up = A B_up^T, then U = Up + E[ids], H = SiLU(G) * U in the
+// epilogue; outputs ep.H and, when not NULL, ep.G and ep.U.  All operands K-major.
+cudaError_t launch_tc_gemm_dagger(int M, int N, int K, const void* A, const void* B_gate, const void* B_up,
+                                  const EpiParams& ep, cudaStream_t stream);
 
 size_t tc_gemm_scratch_bytes();
 

@@ -167,13 +167,13 @@ WORKLOADS = {
     "1b": Workload("1b", 16384, 2048, 8192, 32000, "bf16", "zipf"),
     # long-context forward only, one sequence of 32768 tokens
     "1b_long_fwd": Workload("1b_long_fwd", 32768, 2048, 8192, 32000, "bf16", "mix", backward=False),
-    # 16 independent 1B-class layers, tables in pinned host memory
     # long-context prefill through 16 layers, tables in pinned host memory, optional hot rows on the device
     "1b_prefill_host_x16": Workload("1b_prefill_host_x16", 32768, 2048, 8192, 32000, "bf16", "mix",
                                     backward=False, layers=16, host_tables=True),
     # decode steps: 256 sequences, one new token each per step, table in pinned host memory
     "1b_decode_lfu": Workload("1b_decode_lfu", 256, 2048, 8192, 32000, "bf16", "zipf", backward=False,
                               host_tables=True, note="decode"),
+    # 16 independent 1B-class layers, tables in pinned host memory
     "1b_host_x16": Workload("1b_host_x16", 16384, 2048, 8192, 32000, "bf16", "zipf",
                             layers=16, host_tables=True),
 }

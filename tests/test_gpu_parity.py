@@ -533,11 +533,16 @@ def test_prefetch_with_hot_set_and_prefill_stack():
             assert stack.stats.tolist() == [2 * L * n_hot, 2 * L * (n_u - n_hot)]
 
 
-@pytest.mark.parametrize("dtype_code,flags,tol", [(B.DTYPE_BF16, 0, TOL_BF16), (B.DTYPE_BF16, B.FLAG_SIMT, TOL_BF16),
-                                                   (B.DTYPE_FP32, 0, TOL_FP32)], ids=["tcgen05", "fma_bf16", "fp32"])
-def test_dagger_variant(dtype_code, flags, tol):
-    """STEM-dagger, forward and backward, against the checker (ragged sizes, repeated ids)."""
-    w = synth.Workload("t", 700, 264, 520, 900, "bf16" if dtype_code == B.DTYPE_BF16 else "fp32", "zipf")
+@pytest.mark.parametrize("T,d,F", [(700, 264, 520), (2100, 512, 1160)], ids=["small", "many_tiles"])
+@pytest.mark.parametrize("dtype_code,flags,tol", [(B.DTYPE_BF16, 0, TOL_BF16), (B.DTYPE_BF16, B.FLAG_DAGGER_FUSED, TOL_BF16),
+                                                   (B.DTYPE_BF16, B.FLAG_SINGLE_CTA, TOL_BF16),
+                                                   (B.DTYPE_BF16, B.FLAG_SIMT, TOL_BF16), (B.DTYPE_FP32, 0, TOL_FP32)],
+                         ids=["tcgen05", "tcgen05_two_products_one_launch", "tcgen05_single", "fma_bf16", "fp32"])
+def test_dagger_variant(dtype_code, flags, tol, T, d, F):
+    """STEM-dagger, forward and backward, against the checker (ragged sizes, repeated ids).  With the
+    fused flag the gate and up products share one launch and two accumulators; the other paths run
+    them as two launches."""
+    w = synth.Workload("t", T, d, F, 900, "bf16" if dtype_code == B.DTYPE_BF16 else "fp32", "zipf")
     inp = synth.make_inputs(w, seed=120)
     W_up_np = synth.normal(120, 9, (w.d_ff, w.d_model), w.d_model ** -0.5)
     if dtype_code == B.DTYPE_BF16:
@@ -558,12 +563,17 @@ def test_dagger_variant(dtype_code, flags, tol):
     y_ref, im = O.dagger_forward(inp["x"], inp["ids"], inp["W_gate"], W_up_np, inp["E"], inp["W_down"], True)
     bw = O.dagger_backward(inp["dy"], inp["x"], inp["ids"], inp["W_gate"], W_up_np, inp["E"], inp["W_down"])
     n_u = int(b["n_unique"].item())
-    pairs = {"U": (U, im["U"]), "H": (b["H"], im["H"]), "y": (b["y"], y_ref), "dx": (b["dx"], bw["dx"]),
+    pairs = {"U": (U, im["U"]), "G": (b["G"], im["G"]), "H": (b["H"], im["H"]), "y": (b["y"], y_ref), "dx": (b["dx"], bw["dx"]),
              "dW_gate": (b["dW_gate"], bw["dW_gate"]), "dW_up": (dW_up, bw["dW_up"]),
              "dW_down": (b["dW_down"], bw["dW_down"]), "dE_rows": (b["dE_rows"][:n_u], bw["dE_rows"])}
     errs = {k: _measures(_np(g), r, tol, k in ROWWISE) for k, (g, r) in pairs.items()}
     bad = {k: v for k, v in errs.items() if not v["ok"]}
     assert not bad, (bad, errs)
+    # forward alone, keeping nothing but what the call requires (U): the same y
+    y2 = torch.zeros_like(b["y"])
+    B.stem_dagger_forward(st.shape, st.x, st.ids, st.W_gate, W_up, st.E, st.W_down, y2, None, None, U, b["ws"])
+    torch.cuda.synchronize()
+    assert st.status() == B.OK and torch.equal(y2, b["y"])
 
 
 def test_lfu_cache_tracks_the_most_frequent_ids():
