@@ -713,11 +713,12 @@ cudaError_t launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
 
 struct SecondProduct { int M = 0, N = 0; const void* A = nullptr; const void* B = nullptr; void* out = nullptr; };
 
-template <bool A_MN, bool B_MN, int KIND, int CTAS>
+template <bool A_MN, bool B_MN, int KIND, int CTAS, int BN = 256>
 cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const EpiParams& ep,
                       const SecondProduct& second, cudaStream_t stream) {
   // 192 KB of operand ring either way: 4 stages of 48 KB, or 6 stages of 32 KB per CTA of a pair
-  constexpr int BN = 256, STAGES = CTAS == 2 ? 6 : 4;
+  // (8 stages of 24 KB for the 128-column tiles of decode-sized batches)
+  constexpr int STAGES = BN == 256 ? (CTAS == 2 ? 6 : 4) : (CTAS == 2 ? 8 : 5);
   CUtensorMap tmA, tmB;
   const bool okA = A_MN ? encode_map(&tmA, A, K, M, BK) : encode_map(&tmA, A, M, K, BM);
   const bool okB = B_MN ? encode_map(&tmB, B, K, N, BK) : encode_map(&tmB, B, N, K, BN / CTAS);
@@ -774,6 +775,14 @@ cudaError_t launch_bn(const void* A, const void* B, int M, int N, int K, const E
 template <bool A_MN, bool B_MN, int KIND>
 cudaError_t launch_ctas(const void* A, const void* B, int M, int N, int K, const EpiParams& ep, bool pair,
                         cudaStream_t stream) {
+  if constexpr (KIND == kEpiGate) {
+    // A decode-sized batch (one row of tiles) leaves most CTA pairs without a tile and makes the
+    // one tile a pair has a serial chain of load, multiply, epilogue.  Halving the tile width
+    // doubles the pairs at work and halves that chain; beyond 256 rows the extra passes over x
+    // cost more than they save (measured: 256 rows 22.6 -> 20.5 us, 512 rows 23.8 -> 28.8 us).
+    if (pair && M <= 256 && (N + 127) / 128 <= device_sm_count() / 2)
+      return launch_bn<A_MN, B_MN, KIND, 2, 128>(A, B, M, N, K, ep, SecondProduct{}, stream);
+  }
   if (pair) return launch_bn<A_MN, B_MN, KIND, 2>(A, B, M, N, K, ep, SecondProduct{}, stream);
   return launch_bn<A_MN, B_MN, KIND, 1>(A, B, M, N, K, ep, SecondProduct{}, stream);
 }
