@@ -22,7 +22,7 @@ constexpr int kSegBlk = 64;     // most sorted positions per CTA (the launch pic
 constexpr int kCtasPerSm = 7;   // register budget the kernel is compiled for
 constexpr int kThreads = 128;   // pass 1: one thread per vector of columns
 constexpr int kBatch = 8;       // rows requested before the first is consumed
-constexpr int kFinBatch = 16;    // finishing kernel: partial rows requested before the first is added
+constexpr int kFinBatch = 8;    // finishing kernel: partial rows requested before the first is added
 
 template <typename T> struct Vec;
 template <> struct Vec<float> {
