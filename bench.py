@@ -653,6 +653,7 @@ def run_sharded(args, w):
 
 
 TWO_PRODUCTS = ("dw_pair_gemm", "gate_up_gemm")
+TRAFFIC_SHAPE = (2048, 8192)     # (d_model, d_ff) of the captures behind profiles/ncu_traffic.txt
 NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}   # dense bf16 and HBM3e figures of the data sheet
 
 
@@ -799,9 +800,10 @@ def rooflines(kernels, regime, peaks, T, d, F, bf16):
     roofline = None
     if gemms and bf16:
         dom = min(gemms, key=lambda n: gemms[n]["tflops"])      # the contraction furthest from the peak
-        cap = load_traffic(dom)
-        # DRAM traffic grows in proportion to the tokens of a launch (every [T,.] operand does; the
-        # weights are the small remainder), so a capture at fewer tokens is scaled by T / T_captured.
+        # The stored counters were taken at the 1B-class shape.  DRAM traffic grows in proportion to
+        # the tokens of a launch (every [T,.] operand does; the weights are the small remainder), so
+        # a capture at fewer tokens is scaled by T / T_captured; other shapes have no counters.
+        cap = load_traffic(dom) if (d, F) == TRAFFIC_SHAPE else None
         traffic = cap[1] * T / cap[0] if cap else None
         key = "bf16_tflops" if regime == "burst" else "bf16_tflops_sustained"
         g = gemms[dom]
@@ -816,9 +818,10 @@ def rooflines(kernels, regime, peaks, T, d, F, bf16):
     if hbm:
         worst = min(hbm, key=lambda n: hbm[n]["frac_of_measured_hbm"])
         k = hbm[worst]
+        cap = load_traffic(worst) if (d, F) == TRAFFIC_SHAPE else None
         roofline_hbm = {"kernel": worst, "bound": "hbm", "achieved": k["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": k["frac_of_measured_hbm"], "frac_nominal": k["frac_of_nominal_hbm"],
-                        "bytes_per_launch": k["bytes"], "traffic": None,
+                        "bytes_per_launch": k["bytes"], "traffic": cap[1] * T / cap[0] if cap else None,
                         "peak_source": f"{peaks['source']} (copy bandwidth, of measured); nominal 8000 GB/s",
                         "all": {n: v["frac_of_measured_hbm"] for n, v in hbm.items()}}
     return roofline, roofline_hbm
