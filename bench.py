@@ -193,7 +193,7 @@ def run_reference(args, w):
     }))
 
 
-def run_host_stack(args, w):
+def run_host_stack(args, w, steps=None, warmup=None):
     """Workload with the tables of a stack of independent layers in pinned host memory: a step is
     forward + backward of every layer, rows prefetched and gradient rows written back on side
     streams.  Reports tokens/s (all layers) and the exposed copy time: the time of the same stack
@@ -206,6 +206,8 @@ def run_host_stack(args, w):
     dev = torch.device("cuda", 0)
     B.lib()
     dt = torch.bfloat16
+    steps = args.steps if steps is None else steps
+    warmup = args.warmup if warmup is None else warmup
     T, d, F, V, L = (args.tokens or w.T), w.d_model, w.d_ff, w.V, w.layers
     gcode = B.DTYPE_BF16 if args.grad_bf16 else B.DTYPE_FP32
     gen = torch.Generator(device=dev).manual_seed(args.seed)
@@ -230,7 +232,7 @@ def run_host_stack(args, w):
     results = {}
     for name, resident in (("resident", True), ("host", False)):
         stack = runner.HostTableStack(shape, L, dev_tables if resident else host_tables, W_gate, W_down, resident)
-        for _ in range(args.warmup):
+        for _ in range(warmup):
             stack.step(xs, idss, dys)
         stack.finish()
         torch.cuda.synchronize()
@@ -239,14 +241,14 @@ def run_host_stack(args, w):
         with ClockSampler(0) as clocks:
             t0 = time.time()
             ev0.record(stream)
-            for _ in range(args.steps):
+            for _ in range(steps):
                 stack.step(xs, idss, dys)
             stack.finish()
             ev1.record(stream)
             torch.cuda.synchronize()
             t1 = time.time()
         assert B.stem_query_status(stack.ws) == B.OK
-        results[name] = {"ms": ev0.elapsed_time(ev1) / args.steps, "launches": B.stem_launch_count() - l0,
+        results[name] = {"ms": ev0.elapsed_time(ev1) / steps, "launches": B.stem_launch_count() - l0,
                          "clocks": clocks.summary(t0, t1),
                          "n_unique": [int(k["n_unique"].item()) for k in stack.slots]}
         if not resident:
@@ -288,9 +290,9 @@ def run_host_stack(args, w):
     n_u = float(np.mean(results["host"]["n_unique"]))
     peaks = load_peaks()
     tf = 12.0 * L * T * d * F / (host_ms * 1e-3) / 1e12
-    print(json.dumps({
-        "metric": METRIC, "value": L * T / (host_ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": host_ms, "higher_is_better": True, "scaling": "weak",
+    return {
+        "metric": METRIC, "value": L * T / (host_ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": steps,
+        "warmup": warmup, "ms_per_step": host_ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "layers": L, "T": T, "d_model": d, "d_ff": F, "V": V, "ids": w.id_dist,
                    "tables": "pinned host memory, one per layer", "grad_dtype": "bf16" if args.grad_bf16 else "f32",
@@ -305,7 +307,7 @@ def run_host_stack(args, w):
                      "frac": tf / peaks["bf16_tflops_sustained"], "traffic": None,
                      "peak_source": peaks["source"] + " (sustained bf16 GEMM, of measured)",
                      "kernel": "whole step (six contractions per layer)"},
-    }))
+    }
 
 
 def run_prefill_stack(args, w):
@@ -978,6 +980,8 @@ def main():
     ap.add_argument("--no-profile", action="store_true",
                     help="do not record per-step events inside the timed region (checks what they cost)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
+    ap.add_argument("--no-host-config", action="store_true",
+                    help="default workload only: skip the host-table stack among the other configurations")
     ap.add_argument("--no-configs", action="store_true",
                     help="default workload only: skip the short timings of the other single-layer configurations")
     ap.add_argument("--sharded", action="store_true",
@@ -1012,7 +1016,7 @@ def main():
         if w.note == "decode":
             run_decode(args, w)
         elif w.backward:
-            run_host_stack(args, w)
+            print(json.dumps(run_host_stack(args, w)))
         else:
             run_prefill_stack(args, w)
         return
@@ -1160,6 +1164,15 @@ def main():
                 "tflops_step": layer_flops(wc.T, wc.d_model, wc.d_ff, wc.backward) / (ms_c * 1e-3) / 1e12,
                 "gpu_launches": m["launches"], "clocks": m["clocks"], "roofline": rf, "roofline_hbm": rf_hbm, "kernels": kern}
             del m
+            torch.cuda.empty_cache()
+        if not args.no_host_config:
+            # the host-table configuration: every layer of the stack, three timed passes
+            wh = synth.WORKLOADS["1b_host_x16"]
+            h = run_host_stack(args, wh, steps=3, warmup=3)
+            configs[wh.name] = {k: h[k] for k in ("value", "unit", "steps", "warmup", "ms_per_step", "tflops_step", "config",
+                                                   "gpu_launches", "clocks", "host_tables", "device_tables",
+                                                   "exposed_copy_ms_per_layer", "host_link", "rows_prefetched_per_layer",
+                                                   "prefetch_bytes_per_layer", "writeback_bytes_per_layer")}
             torch.cuda.empty_cache()
 
     out = {
