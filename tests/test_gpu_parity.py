@@ -219,6 +219,40 @@ def test_randomized_shapes_layouts_and_gradient_types():
             raise AssertionError(f"case {case}: T={T} d={d} F={F} V={V} {dist} flags={flags} grad={grad}: {e}") from e
 
 
+@pytest.mark.parametrize("flags", [0, B.FLAG_SIMT], ids=["tcgen05", "fma"])
+def test_backward_with_outputs_left_out(flags):
+    """Any of dx, dW_gate, dW_down, dE_rows may be NULL: the outputs that are asked for equal those
+    of the full call (dx and the table-gradient rows bit for bit; the weight gradients to fp32
+    rounding, since the two share a launch, and with it possibly a different split of the token
+    range, only when both are asked for), and the others are not touched."""
+    w = synth.Workload("t", 2304, 264, 520, 700, "bf16", "zipf")
+    st = runner.state_from_numpy(synth.make_inputs(w, seed=83), B.DTYPE_BF16, w.V, flags=flags)
+    st.step()
+    torch.cuda.synchronize()
+    b = st.bufs
+    n_u = int(b["n_unique"].item())
+    names = ("dx", "dW_gate", "dW_down", "dE_rows")
+    full = {k: b[k].clone() for k in names}
+    for keep in (("dx",), ("dW_gate",), ("dW_down",), ("dE_rows",), ("dW_gate", "dW_down"), ("dx", "dE_rows"), ()):
+        for k in names:
+            b[k].fill_(3.0)
+        args = {k: (b[k] if k in keep else None) for k in names}
+        B.stem_ffn_backward(st.shape, st.dy, st.x, st.ids, st.W_gate, st.E, st.W_down, b["G"], b["H"], b["perm"],
+                            b["seg_offsets"], b["n_unique"], args["dx"], args["dW_gate"], args["dW_down"], args["dE_rows"],
+                            b["unique_ids"], b["ws"])
+        torch.cuda.synchronize()
+        assert st.status() == B.OK
+        for k in names:
+            if k in keep:
+                got, ref = (b[k][:n_u], full[k][:n_u]) if k == "dE_rows" else (b[k], full[k])
+                if k in ("dx", "dE_rows"):
+                    assert torch.equal(got, ref), (keep, k)
+                else:
+                    assert float((got - ref).abs().max()) <= 1e-5 * float(ref.abs().max()), (keep, k)
+            else:
+                assert bool((b[k] == 3.0).all()), (keep, k)
+
+
 def test_backward_is_bitwise_reproducible():
     w = synth.Workload("t", 2048, 256, 1024, 500, "bf16", "zipf")
     st = runner.state_from_numpy(synth.make_inputs(w, seed=79), B.DTYPE_BF16, w.V)
