@@ -53,6 +53,8 @@ def test_gemm_layouts(flags, a_mn, b_mn, M, N, K):
     ("uniform", 256, 4096), ("zipf", 16384, 32000), ("mix", 32768, 32000), ("same", 1000, 77),
     ("distinct", 3000, 5000), ("uniform", 1, 5), ("uniform", 70001, 300), ("zipf", 100000, 1 << 20),
     ("uniform", 65, 2), ("uniform", 4097, 1), ("zipf", 1024, 500), ("zipf", 1025, 500), ("same", 1024, 9),
+    ("uniform", 65536, 70000), ("zipf", 65537, 32000), ("distinct", 40000, 40000), ("same", 50000, 3),
+    ("uniform", 2049, 1 << 26),
 ])
 def test_dedup_bit_exact(dist, T, V):
     ids = synth.token_ids(5, T, V, dist)
@@ -95,6 +97,35 @@ def test_dedup_largest_supported_batch():
         assert np.array_equal(b[k][:n].cpu().numpy(), ref[k]), k
 
 
+def test_dedup_one_workspace_many_batches():
+    """Batches of different lengths, one after another with no host synchronisation between them, through
+    one workspace: nothing a call leaves in the sort's scratch (keys, digit counts, head counts of a longer
+    or shorter batch, of 1, 2, 16, 64 or 69 CTAs) may reach the next call's outputs."""
+    V = 32000
+    sizes = [700, 1025, 65536, 70000, 16384, 1500, 65536, 3]
+    big = B.make_shape(max(sizes), 8, 8, V, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+    ws = torch.empty(B.stem_workspace_bytes(big), dtype=torch.uint8, device="cuda")
+    B.stem_init_workspace(ws)
+    outs, refs = [], []
+    for k, T in enumerate(sizes):
+        ids = synth.token_ids(40 + k, T, V, ("zipf", "uniform", "mix")[k % 3])
+        refs.append(O.dedup(ids))
+        R = min(T, V)
+        o = {"ids": torch.from_numpy(ids).cuda(), "T": T}
+        for name, n in (("unique_ids", R), ("n_unique", 1), ("inverse", T), ("perm", T), ("seg_offsets", R + 1)):
+            o[name] = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        outs.append(o)
+    for o in outs:                                              # all launches first, then one sync
+        shp = B.make_shape(o["T"], 8, 8, V, B.DTYPE_BF16, B.DTYPE_FP32, 0)
+        B.stem_dedup_ids(shp, o["ids"], o["unique_ids"], o["n_unique"], o["inverse"], o["perm"], o["seg_offsets"], ws)
+    assert B.stem_query_status(ws) == B.OK
+    for o, ref in zip(outs, refs):
+        n_u = int(o["n_unique"].item())
+        assert n_u == ref["n_unique"]
+        for name, n in (("unique_ids", n_u), ("perm", o["T"]), ("seg_offsets", n_u + 1), ("inverse", o["T"])):
+            assert np.array_equal(o[name][:n].cpu().numpy(), ref[name]), (o["T"], name)
+
+
 def test_layer_many_tokens_narrow():
     """A long batch (131072 positions, several hundred row tiles) on a narrow layer: every tile row
     of the token dimension, ragged d_ff, heavy id repetition."""
@@ -116,6 +147,15 @@ def test_dedup_empty_and_bad_ids():
     assert np.array_equal(st.bufs["perm"][:5].cpu().numpy(), ref["perm"])
     B.stem_init_workspace(st.bufs["ws"])
     assert st.status() == B.OK
+    ids = synth.token_ids(6, 3000, 10, "uniform")             # the same through the radix path
+    ids[17], ids[2999] = 10, -1
+    st = runner.LayerState(B.make_shape(3000, 8, 8, 10, B.DTYPE_BF16, B.DTYPE_FP32, 0)).allocate(backward=False)
+    st.ids = torch.from_numpy(ids).cuda()
+    st.dedup()
+    assert st.status() == B.ERR_ID_RANGE
+    ref = O.dedup(np.clip(ids, 0, 9))
+    assert np.array_equal(st.bufs["perm"][:3000].cpu().numpy(), ref["perm"])
+    assert np.array_equal(st.bufs["inverse"][:3000].cpu().numpy(), ref["inverse"])
 
 
 # ---------------------------------------------------------------------------------------
